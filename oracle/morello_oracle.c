@@ -1,0 +1,182 @@
+/*
+ * CPU oracle for MatmulAccum  --  TEST INFRASTRUCTURE, NOT THE PRODUCT.
+ *
+ * Only the tests, the smoke check and the benchmark's cpu_baseline / reference
+ * leg may call this file.  It shares no code with the CUDA library and is
+ * never a fallback for it.
+ *
+ * What it computes (paper Section 2, "Tiling": dimensions are ordered
+ * batch, m, k, n and the output is batch x m x n; Section 2.2: the
+ * accumulating primitive MatmulAccum adds into the existing contents of its
+ * output, and the operand types are bf16, bf16 -> f32; Section 2.2 item 3 on
+ * Move: a bf16 -> f32 move is an upcast copy, i.e. the inputs are widened
+ * exactly before they are multiplied):
+ *
+ *     C[b,i,j]  <-  C[b,i,j] + sum_{p=0}^{k-1} A[b,i,p] * B[b,p,j]
+ *
+ * Layout: dense row-major A[b][m][k], B[b][k][n] (bf16 bit patterns in
+ * uint16_t), C[b][m][n] (float).
+ *
+ * Precision: the paper fixes no summation order (Section 2: the iteration
+ * order of a tile loop is undefined), so the oracle is the plain definition:
+ * start from (double)C, add the exact products (a bf16 x bf16 product has at
+ * most 16 significant bits, exact in double) for p = 0..k-1 in increasing
+ * order in double, and round ONCE to float (round-to-nearest-even, the C
+ * default) at the end.
+ *
+ * Pins (tests/test_oracle_pins.py): exact rational brute force on tiny
+ * shapes, closed forms, identity / zero / one-hot operands, the accumulate
+ * invariant, integer exactness against integer matrix products, power-of-two
+ * scaling, and agreement with a float64 library contraction.
+ * NaN / Inf / subnormal inputs: parity unpinned (they follow IEEE through the
+ * C arithmetic below; no test fixes their behaviour).
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <math.h>
+
+/* bf16 is the upper 16 bits of an IEEE binary32: widening is a 16-bit shift. */
+static inline double bf16_to_double(uint16_t h)
+{
+    uint32_t u = ((uint32_t)h) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/*
+ * The definition, written as the literal triple loop (b, i, j, p).
+ * Serial; meant for small shapes.
+ */
+void oracle_matmul_accum_naive(int64_t b, int64_t m, int64_t k, int64_t n,
+                               const uint16_t *A, const uint16_t *B, float *C)
+{
+    for (int64_t bb = 0; bb < b; ++bb)
+        for (int64_t i = 0; i < m; ++i)
+            for (int64_t j = 0; j < n; ++j) {
+                double s = (double)C[(bb * m + i) * n + j];
+                for (int64_t p = 0; p < k; ++p)
+                    s += bf16_to_double(A[(bb * m + i) * k + p]) *
+                         bf16_to_double(B[(bb * k + p) * n + j]);
+                C[(bb * m + i) * n + j] = (float)s;
+            }
+}
+
+/*
+ * One output row (bb, i), all n columns: the same arithmetic per element in
+ * the same p order as the triple loop, with the j loop innermost so that B is
+ * walked along its rows.  `s` is a caller-provided buffer of n doubles.
+ * If T is not NULL it receives sum_p |A[b,i,p] * B[b,p,j]| (the scale of the
+ * floating-point tolerance) for the row.
+ */
+static void oracle_row(int64_t bb, int64_t i, int64_t m, int64_t k, int64_t n,
+                       const uint16_t *A, const uint16_t *B,
+                       const float *Cin_row, float *Cout_row, double *T_row,
+                       double *s)
+{
+    for (int64_t j = 0; j < n; ++j) s[j] = (double)Cin_row[j];
+    if (T_row) for (int64_t j = 0; j < n; ++j) T_row[j] = 0.0;
+    for (int64_t p = 0; p < k; ++p) {
+        const double a = bf16_to_double(A[(bb * m + i) * k + p]);
+        const uint16_t *Brow = B + (bb * k + p) * n;
+        for (int64_t j = 0; j < n; ++j) s[j] += a * bf16_to_double(Brow[j]);
+        if (T_row)
+            for (int64_t j = 0; j < n; ++j)
+                T_row[j] += fabs(a * bf16_to_double(Brow[j]));
+    }
+    for (int64_t j = 0; j < n; ++j) Cout_row[j] = (float)s[j];
+}
+
+/*
+ * Whole problem, in place on C.  Rows (b, i) are independent, so they are
+ * handed to host threads (OpenMP) when the library is built with -fopenmp;
+ * the arithmetic of every element is unchanged by the threading.
+ * Returns 0, or -1 if the scratch row could not be allocated.
+ */
+int oracle_matmul_accum(int64_t b, int64_t m, int64_t k, int64_t n,
+                        const uint16_t *A, const uint16_t *B, float *C)
+{
+    if (b <= 0 || m <= 0 || n <= 0) return 0;
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *s = (double *)malloc((size_t)n * sizeof(double));
+        if (!s) {
+#pragma omp atomic write
+            failed = 1;
+        } else {
+#pragma omp for schedule(dynamic, 1)
+            for (int64_t r = 0; r < b * m; ++r) {
+                float *row = C + r * n;
+                oracle_row(r / m, r % m, m, k, n, A, B, row, row, NULL, s);
+            }
+        }
+        free(s);
+    }
+    return failed ? -1 : 0;
+}
+
+/*
+ * Selected rows only (for checking samples of a large problem and for timing
+ * a bounded sample): rows[t] = bb * m + i.  C_in is the full input C and is
+ * not modified; out[t][0..n) receives the result row; T (nrows x n doubles,
+ * may be NULL) receives sum_p |A*B| for those rows.
+ */
+int oracle_matmul_accum_rows(int64_t b, int64_t m, int64_t k, int64_t n,
+                             const uint16_t *A, const uint16_t *B,
+                             const float *C_in, int64_t nrows,
+                             const int64_t *rows, float *out, double *T)
+{
+    if (n <= 0 || nrows <= 0) return 0;
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *s = (double *)malloc((size_t)n * sizeof(double));
+        if (!s) {
+#pragma omp atomic write
+            failed = 1;
+        } else {
+#pragma omp for schedule(dynamic, 1)
+            for (int64_t t = 0; t < nrows; ++t) {
+                const int64_t r = rows[t];
+                if (r < 0 || r >= b * m) continue;
+                oracle_row(r / m, r % m, m, k, n, A, B, C_in + r * n,
+                           out + t * n, T ? T + t * n : NULL, s);
+            }
+        }
+        free(s);
+    }
+    return failed ? -1 : 0;
+}
+
+/*
+ * T[b,i,j] = sum_p |A[b,i,p] * B[b,p,j]| in double: the magnitude the
+ * floating-point acceptance rule scales with
+ * (|gpu - oracle| <= 1e-5 * T + 1e-6).
+ */
+void oracle_abs_dot(int64_t b, int64_t m, int64_t k, int64_t n,
+                    const uint16_t *A, const uint16_t *B, double *T)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < b * m; ++r) {
+        const int64_t bb = r / m, i = r % m;
+        double *Trow = T + r * n;
+        for (int64_t j = 0; j < n; ++j) Trow[j] = 0.0;
+        for (int64_t p = 0; p < k; ++p) {
+            const double a = bf16_to_double(A[(bb * m + i) * k + p]);
+            const uint16_t *Brow = B + (bb * k + p) * n;
+            for (int64_t j = 0; j < n; ++j)
+                Trow[j] += fabs(a * bf16_to_double(Brow[j]));
+        }
+    }
+}
+
+#ifdef _OPENMP
+#include <omp.h>
+int oracle_num_threads(void) { return omp_get_max_threads(); }
+void oracle_set_num_threads(int t) { if (t > 0) omp_set_num_threads(t); }
+#else
+int oracle_num_threads(void) { return 1; }
+void oracle_set_num_threads(int t) { (void)t; }
+#endif

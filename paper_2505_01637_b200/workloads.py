@@ -1,0 +1,156 @@
+"""Seeded synthetic inputs for MatmulAccum.
+
+This module holds data generation only -- none of the method's arithmetic --
+so that the CPU oracle's tests and the CUDA path's tests can both draw the
+same tensors from it.  It imports numpy and nothing else from this project.
+
+The paper's workloads are dense matrix multiplies with no dataset: the shapes
+are the ones it names (Figure 1: b,m,k,n = 1,4,4,16; Section 7: the
+1 x 2048 x 16384 bf16 -> f32 vector-matrix multiply), widened with a skinny
+decode-style batch, a square GEMM and a large batched GEMM.  Its gemma.cpp
+integration used model weights; the tensors drawn here stand in for them.
+
+Recipe: ``rng = numpy.random.Generator(numpy.random.Philox(seed))`` with
+``seed = 1000 * c + beta`` for config index c (0-based) and batch beta; A[beta],
+then B[beta], then C[beta] are drawn in that order, row-major, as f32; A and B
+are then rounded once to bf16 (round-to-nearest-even, integer arithmetic on the
+f32 bit pattern).  Integer variants use ``seed + 500``.
+"""
+from __future__ import annotations
+
+import zlib
+from dataclasses import dataclass
+
+import numpy as np
+
+
+@dataclass(frozen=True)
+class Config:
+    name: str
+    b: int
+    m: int
+    k: int
+    n: int
+    ab: str          # distribution of A and B: "uniform", "uniform_rsqrtk", "normal_rsqrtk"
+    c: str           # distribution of C: "zeros", "normal", "normal0.1"
+    note: str
+
+    @property
+    def shape(self):
+        return (self.b, self.m, self.k, self.n)
+
+    @property
+    def macs(self):
+        return self.b * self.m * self.k * self.n
+
+    @property
+    def flops(self):
+        return 2 * self.macs
+
+    @property
+    def algorithmic_bytes(self):
+        """A and B read once, C read once and written once."""
+        b, m, k, n = self.shape
+        return 2 * b * m * k + 2 * b * k * n + 2 * 4 * b * m * n
+
+
+CONFIGS = (
+    Config("cfg1_figure1", 1, 4, 4, 16, "uniform", "normal",
+           "Figure 1 shape"),
+    Config("cfg2_gemv", 1, 1, 2048, 16384, "uniform", "zeros",
+           "Section 7 vector-matrix multiply, HBM-bound"),
+    Config("cfg3_skinny16", 1, 16, 2048, 16384, "uniform_rsqrtk", "normal",
+           "decode-style batch, GEMV/GEMM crossover"),
+    Config("cfg4_square4096", 1, 4096, 4096, 4096, "normal_rsqrtk", "zeros",
+           "square GEMM, tensor-core bound"),
+    Config("cfg5_batched", 8, 2048, 2048, 16384, "normal_rsqrtk", "normal0.1",
+           "large batched GEMM with fused accumulate epilogue"),
+)
+
+
+def f32_to_bf16_rne(x: np.ndarray) -> np.ndarray:
+    """Round f32 to bf16 bit patterns (uint16), ties to even; finite inputs."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    bias = np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))
+    return ((u + bias) >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_to_f32(h: np.ndarray) -> np.ndarray:
+    """Widen bf16 bit patterns (uint16) to f32 exactly."""
+    return (np.ascontiguousarray(h, dtype=np.uint16).astype(np.uint32)
+            << np.uint32(16)).view(np.float32)
+
+
+def _draw_ab(rng, shape, dist, k):
+    if dist == "uniform":
+        x = rng.random(shape, dtype=np.float32) * np.float32(2) - np.float32(1)
+    elif dist == "uniform_rsqrtk":
+        x = rng.random(shape, dtype=np.float32) * np.float32(2) - np.float32(1)
+        x *= np.float32(1.0 / np.sqrt(k))
+    elif dist == "normal_rsqrtk":
+        x = rng.standard_normal(shape, dtype=np.float32)
+        x *= np.float32(1.0 / np.sqrt(k))
+    elif dist == "int4":
+        x = rng.integers(-4, 5, size=shape).astype(np.float32)
+    else:
+        raise ValueError(dist)
+    return f32_to_bf16_rne(x)
+
+
+def _draw_c(rng, shape, dist):
+    if dist == "zeros":
+        return np.zeros(shape, dtype=np.float32)
+    if dist == "normal":
+        return rng.standard_normal(shape, dtype=np.float32)
+    if dist == "normal0.1":
+        return rng.standard_normal(shape, dtype=np.float32) * np.float32(0.1)
+    if dist == "int8":
+        return rng.integers(-8, 9, size=shape).astype(np.float32)
+    raise ValueError(dist)
+
+
+def make(b, m, k, n, seed, ab="uniform", c="normal"):
+    """(A, B, C) for an arbitrary shape: A, B uint16 bf16 patterns, C f32.
+
+    Batch beta is drawn from Philox(seed + beta): A, then B, then C."""
+    A = np.empty((b, m, k), dtype=np.uint16)
+    B = np.empty((b, k, n), dtype=np.uint16)
+    C = np.empty((b, m, n), dtype=np.float32)
+    for beta in range(b):
+        rng = np.random.Generator(np.random.Philox(seed + beta))
+        A[beta] = _draw_ab(rng, (m, k), ab, max(k, 1))
+        B[beta] = _draw_ab(rng, (k, n), ab, max(k, 1))
+        C[beta] = _draw_c(rng, (m, n), c)
+    return A, B, C
+
+
+def make_config(index: int, variant: str = "random"):
+    """Inputs of BASELINE config ``index`` (0-based).
+
+    variant: "random" (the config's own distributions), "integer" (A, B integer
+    uniform in [-4, 4], C as the config says) or "integer_intc" (C integers in
+    [-8, 8] as well)."""
+    cfg = CONFIGS[index]
+    b, m, k, n = cfg.shape
+    if variant == "random":
+        return make(b, m, k, n, 1000 * index, cfg.ab, cfg.c)
+    if variant == "integer":
+        return make(b, m, k, n, 1000 * index + 500, "int4", cfg.c)
+    if variant == "integer_intc":
+        return make(b, m, k, n, 1000 * index + 500, "int4", "int8")
+    raise ValueError(variant)
+
+
+def crc32(x: np.ndarray) -> int:
+    return zlib.crc32(np.ascontiguousarray(x).view(np.uint8).reshape(-1).data) & 0xFFFFFFFF
+
+
+def sample_rows(b, m, seed, edge=128, per_batch=32):
+    """Flattened row ids (bb*m + i): the first and last ``edge`` rows of batch 0
+    plus ``per_batch`` seeded random rows of every batch (sorted, unique)."""
+    rng = np.random.Generator(np.random.Philox(seed))
+    rows = set(range(min(edge, m))) | set(range(max(0, m - edge), m))
+    for beta in range(b):
+        for i in rng.integers(0, m, size=min(per_batch, m)):
+            rows.add(beta * m + int(i))
+    return np.array(sorted(rows), dtype=np.int64)
