@@ -1,0 +1,476 @@
+#!/usr/bin/env python
+"""Benchmark of the B200 MatmulAccum library (bf16 x bf16 -> f32, accumulating).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--configs 1,3,4,5] [--no-cpu-baseline]
+
+One JSON line on stdout.  A step is one MatmulAccum call on the headline
+workload, the 1 x 2048 x 16384 vector-matrix multiply: `value` is its
+algorithmic bytes (A and B read once, C read and written once) per second with
+all operands resident in HBM; the B matrix rotates over 8 distinct 64 MiB
+buffers so that no call finds its input in L2.  `e2e` is the same metric
+through the host-buffer entry point, host<->device copies inside the timed
+region.  `configs` reports the other shapes (GEMM ones in TFLOP/s), each
+against its own roofline.  With --gpus N every rank runs an independent replica
+(the operation has no exchange step); the time is the maximum over ranks.
+
+--impl reference times the CPU oracle (the only baseline there is: the paper
+ships no code) on this machine's host cores, on a bounded sample of the same
+workload."""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2505_01637_b200 import workloads as w
+
+METRIC = "bf16->f32 MatmulAccum: GEMV HBM GB/s & GEMM TFLOP/s, % of B200 roofline"
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+HEADLINE = 1            # index into workloads.CONFIGS: the 1 x 2048 x 16384 GEMV
+ROTATE = 8              # distinct B buffers: 8 x 64 MiB = 512 MiB > 4 x the 126 MB L2
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def load_traffic():
+    """DRAM bytes per launch from the committed ncu summaries (None if absent)."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        return json.load(open(path))
+    except Exception:
+        return {}
+
+
+# ------------------------------------------------------------------ clock sampler
+class ClockSampler:
+    """Samples SM clock and clock-event reasons through NVML (read-only) while
+    the timed regions run."""
+
+    def __init__(self, index: int):
+        self.samples = []          # (t, sm_mhz, reasons_bitmask, power_w)
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _loop(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                mhz = int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    reasons = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    reasons = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                try:
+                    power = nv.nvmlDeviceGetPowerUsage(self._h) / 1000.0
+                except Exception:
+                    power = None
+                self.samples.append((time.perf_counter(), mhz, reasons, power))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+
+    def summary(self, windows):
+        """Median clock and the reasons seen inside the (t0, t1) windows."""
+        names = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+                 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+                 0x2: "applications_clocks_setting", 0x10: "sync_boost",
+                 0x100: "display_clock_setting"}
+        inside = [s for s in self.samples if any(t0 <= s[0] <= t1 for (t0, t1) in windows)]
+        use = inside or self.samples
+        if not use:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        mask = 0
+        for s in use:
+            mask |= s[2]
+        powers = [s[3] for s in use if s[3] is not None]
+        return {"sm_mhz": statistics.median(s[1] for s in use), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(names[b] for b in names if mask & b),
+                "samples": len(use), "samples_in_timed_regions": len(inside),
+                "power_w_max": max(powers) if powers else None}
+
+
+def nvml_index(local: int) -> int:
+    """NVML index of this rank's GPU (CUDA_VISIBLE_DEVICES may renumber devices)."""
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+    ids = [v.strip() for v in vis.split(",") if v.strip()]
+    if local < len(ids) and ids[local].isdigit():
+        return int(ids[local])
+    return local
+
+
+# ---------------------------------------------------------------- reference arm
+def oracle_sample(cfg_index, budget_s=8.0, threads=None):
+    """Times the CPU oracle, as it stands, on a bounded sample of a config.
+    Returns (seconds, macs, description, threads)."""
+    import oracle
+    if threads:
+        oracle.set_num_threads(threads)
+    cfg = w.CONFIGS[cfg_index]
+    b, m, k, n = cfg.shape
+    if cfg.macs <= 2e9:                       # whole problem per repetition
+        A, B, C = w.make_config(cfg_index)
+        oracle.matmul_accum(b, m, k, n, A, B, C)                     # page in, spin up threads
+        reps, t0 = 0, time.perf_counter()
+        while True:
+            oracle.matmul_accum(b, m, k, n, A, B, C)
+            reps += 1
+            el = time.perf_counter() - t0
+            if el >= budget_s or reps >= 2000:
+                break
+        return el / reps, cfg.macs, "whole problem, mean of %d repetitions" % reps, oracle.num_threads()
+    # a row sample of one batch of a large problem
+    A, B, C = w.make(1, m, k, n, 1000 * cfg_index, cfg.ab, cfg.c)
+    nrows = max(oracle.num_threads(), int(8e9 // (k * n)))
+    rows = np.linspace(0, m - 1, num=min(nrows, m)).astype(np.int64)
+    t0 = time.perf_counter()
+    oracle.matmul_accum_rows(1, m, k, n, A, B, C, rows, want_abs=False)
+    el = time.perf_counter() - t0
+    return el, len(rows) * k * n, "%d of %d rows of batch 0, all columns" % (len(rows), b * m), oracle.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    cfg = w.CONFIGS[HEADLINE]
+    import oracle
+    oracle.build()
+    b, m, k, n = cfg.shape
+    A, B, C = w.make_config(HEADLINE)
+    for _ in range(max(args.warmup, 1)):
+        oracle.matmul_accum(b, m, k, n, A, B, C)
+    steps = max(1, min(args.steps, 200))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.matmul_accum(b, m, k, n, A, B, C)
+    el = time.perf_counter() - t0
+    gbs = cfg.algorithmic_bytes * steps / el / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s",
+        "n_gpus": args.gpus, "steps": steps, "warmup": max(args.warmup, 1),
+        "ms_per_step": el / steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "%s b,m,k,n=%s" % (cfg.name, list(cfg.shape)),
+                   "note": "CPU oracle (double accumulation) on the host cores; each step is "
+                           "the whole vector-matrix multiply"},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": oracle.num_threads(),
+                         "kind": "oracle", "sample": "whole problem per step, %d steps" % steps},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------ GPU arm
+def time_calls(torch, fn, steps, warmup):
+    """fn(i) enqueues step i on the current stream; returns seconds for `steps` steps."""
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    start = torch.cuda.Event(enable_timing=True)
+    stop = torch.cuda.Event(enable_timing=True)
+    start.record()
+    for i in range(steps):
+        fn(i)
+    stop.record()
+    torch.cuda.synchronize()
+    return start.elapsed_time(stop) * 1e-3
+
+
+def bench_config(torch, mb, idx, iters, warmup, peaks, windows, path=None):
+    """Device-timed throughput of one config (inputs resident, rotating when small)."""
+    cfg = w.CONFIGS[idx]
+    b, m, k, n = cfg.shape
+    in_bytes = 2 * b * m * k + 2 * b * k * n + 4 * b * m * n
+    sets = max(1, min(ROTATE, int(np.ceil(512 * 2 ** 20 / in_bytes))))
+    A, B, C = w.make_config(idx)
+    dev = []
+    for s in range(sets):
+        if s == 0:
+            As, Bs = A, B
+        else:                                   # fresh values for every rotating copy
+            As, Bs, _ = w.make(b, m, k, n, 1000 * idx + 100 * s, cfg.ab, "zeros")
+        dev.append((torch.from_numpy(As.view(np.int16)).cuda(), torch.from_numpy(Bs.view(np.int16)).cuda(),
+                    torch.from_numpy(C.copy()).cuda()))
+    ptrs = [(a.data_ptr(), bb.data_ptr(), c.data_ptr()) for (a, bb, c) in dev]
+    stream = torch.cuda.current_stream().cuda_stream
+    call = mb.lib().morello_matmul_accum_forced
+    forced = mb.MORELLO_PATH_AUTO if path is None else path
+
+    def step(i):
+        pa, pb, pc = ptrs[i % sets]
+        rc = call(forced, 0, b, m, k, n, pa, pb, pc, None, 0, stream)
+        if rc != 0:
+            raise mb.MorelloError(rc, "bench %s" % cfg.name)
+
+    l0 = mb.morello_launch_count()
+    step(0)
+    per_call = mb.morello_launch_count() - l0
+    t0 = time.perf_counter()
+    sec = time_calls(torch, step, iters, warmup)
+    windows.append((t0, time.perf_counter()))
+    st, detail = mb.morello_read_device_status()
+    if st != 0:
+        raise RuntimeError("device status %d (0x%x) after %s" % (st, detail, cfg.name))
+    us = sec / iters * 1e6
+    gbs = cfg.algorithmic_bytes / (sec / iters) / 1e9
+    tfl = cfg.flops / (sec / iters) / 1e12
+    chosen = mb.morello_select_path(b, m, k, n) if path is None else path
+    rec = {"name": cfg.name, "shape": list(cfg.shape), "path": "tcgen05" if chosen == 1 else "skinny",
+           "us_per_call": us, "GBps": gbs, "TFLOPs": tfl, "iters": iters, "launches_per_call": per_call,
+           "rotating_sets": sets,
+           "frac_hbm_measured": gbs / peaks["hbm_gbs"], "frac_hbm_nominal": gbs / NOMINAL_HBM_GBS,
+           "frac_tensor_measured_burst": tfl / peaks["bf16_tflops"],
+           "frac_tensor_measured_sustained": tfl / peaks["bf16_tflops_sustained"],
+           "frac_tensor_nominal": tfl / NOMINAL_BF16_TFLOPS}
+    del dev
+    torch.cuda.empty_cache()
+    return rec
+
+
+def run_ours(args):
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    from paper_2505_01637_b200 import binding as mb
+    mb.lib()                                    # raises if the CUDA library is not built
+    peaks, peak_kind = load_peaks()
+    traffic = load_traffic()
+    sampler = ClockSampler(nvml_index(local))
+    windows = []
+
+    cfg = w.CONFIGS[HEADLINE]
+    b, m, k, n = cfg.shape
+    A, B0, C = w.make_config(HEADLINE)
+    host_B = [B0] + [w.make(b, m, k, n, 1000 * HEADLINE + 100 * s, cfg.ab, "zeros")[1]
+                     for s in range(1, ROTATE)]
+    dA = torch.from_numpy(A.view(np.int16)).cuda()
+    dB = [torch.from_numpy(x.view(np.int16)).cuda() for x in host_B]
+    dC = [torch.from_numpy(C.copy()).cuda() for _ in range(ROTATE)]
+    stream = torch.cuda.current_stream().cuda_stream
+    call = mb.lib().morello_matmul_accum
+    pa = dA.data_ptr()
+    pbs = [x.data_ptr() for x in dB]
+    pcs = [x.data_ptr() for x in dC]
+
+    def step(i):
+        rc = call(b, m, k, n, pa, pbs[i % ROTATE], pcs[i % ROTATE], stream)
+        if rc != 0:
+            raise mb.MorelloError(rc, "bench step")
+
+    sampler.start()
+    # ---- headline: K steps, device-timed, barrier + synchronize on both sides
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+        torch.cuda.synchronize()
+    l0 = mb.morello_launch_count()
+    start = torch.cuda.Event(enable_timing=True)
+    stop = torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    start.record()
+    for i in range(args.steps):
+        step(i)
+    stop.record()
+    torch.cuda.synchronize()
+    windows.append((t0, time.perf_counter()))
+    if dist is not None:
+        dist.barrier()
+        torch.cuda.synchronize()
+    launches = mb.morello_launch_count() - l0
+    sec = start.elapsed_time(stop) * 1e-3
+    if dist is not None:
+        t = torch.tensor([sec], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        sec = float(t.item())
+    st, detail = mb.morello_read_device_status()
+    if st != 0:
+        raise RuntimeError("device status %d (0x%x)" % (st, detail))
+    value = world * cfg.algorithmic_bytes * args.steps / sec / 1e9
+
+    # ---- the same loop replayed from a CUDA graph (launch overhead taken out)
+    graph_us = None
+    try:
+        side = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            cap = side.cuda_stream
+            with torch.cuda.graph(g, stream=side):
+                for i in range(ROTATE):
+                    rc = call(b, m, k, n, pa, pbs[i], pcs[i], cap)
+                    assert rc == 0, rc
+            reps = max(1, args.steps // ROTATE)
+            for _ in range(3):
+                g.replay()
+            side.synchronize()
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            t0 = time.perf_counter()
+            e0.record(side)
+            for _ in range(reps):
+                g.replay()
+            e1.record(side)
+            side.synchronize()
+            windows.append((t0, time.perf_counter()))
+            graph_us = e0.elapsed_time(e1) * 1e3 / (reps * ROTATE)
+    except Exception as exc:                     # a diagnostic extra, never fatal
+        graph_us = "failed: %s" % exc
+        torch.cuda.synchronize()
+
+    # ---- end to end through the host-buffer entry point (pinned host memory)
+    hA = torch.from_numpy(A.view(np.int16)).pin_memory()
+    hB = [torch.from_numpy(x.view(np.int16)).pin_memory() for x in host_B[:2]]
+    hC = torch.from_numpy(C.copy()).pin_memory()
+    host_call = mb.lib().morello_matmul_accum_host
+    e2e_steps = max(3, min(args.steps, 30))
+    for i in range(3):
+        assert host_call(b, m, k, n, hA.data_ptr(), hB[i % 2].data_ptr(), hC.data_ptr()) == 0
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        assert host_call(b, m, k, n, hA.data_ptr(), hB[i % 2].data_ptr(), hC.data_ptr()) == 0
+    e2e_sec = time.perf_counter() - t0        # the call returns only when C is back on the host
+    windows.append((t0, time.perf_counter()))
+    if dist is not None:
+        t = torch.tensor([e2e_sec], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_sec = float(t.item())
+    e2e_value = world * cfg.algorithmic_bytes * e2e_steps / e2e_sec / 1e9
+    h2d = 2 * b * m * k + 2 * b * k * n + 4 * b * m * n
+    d2h = 4 * b * m * n
+
+    # ---- the other configurations (rank 0 of a single-GPU run only)
+    extra = []
+    if world == 1 and args.configs:
+        plan = {0: (1000, 50), 2: (300, 20), 3: (30, 5), 4: (6, 2)}
+        for idx in args.configs:
+            if idx == HEADLINE or idx not in plan:
+                continue
+            iters, wu = plan[idx]
+            extra.append(bench_config(torch, mb, idx, iters, wu, peaks, windows))
+            if idx == 2 and mb.morello_select_path(*w.CONFIGS[2].shape) == mb.MORELLO_PATH_SKINNY:
+                try:                            # crossover config: also on the tensor-core path
+                    extra.append(bench_config(torch, mb, idx, iters, wu, peaks, windows,
+                                              path=mb.MORELLO_PATH_TCGEN05))
+                except mb.MorelloError:
+                    pass
+    sampler.stop()
+    clocks = sampler.summary(windows)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sec_cpu, macs, what, threads = oracle_sample(HEADLINE)
+        cpu = {"value": cfg.algorithmic_bytes * (macs / cfg.macs) / sec_cpu / 1e9, "unit": "GB/s",
+               "cores": threads, "kind": "oracle", "sample": what, "seconds_per_step": sec_cpu}
+
+    if rank == 0:
+        per_launch_gbs = cfg.algorithmic_bytes * args.steps / (sec * 1e9)
+        line = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec / args.steps * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "%s b,m,k,n=%s bf16 x bf16 -> f32 accumulate" % (cfg.name, list(cfg.shape)),
+                       "l2": "B rotates over %d distinct 64 MiB buffers (512 MiB > 4 x L2), no flush needed" % ROTATE,
+                       "inputs": "A,B uniform[-1,1) bf16, C zeros; Philox seeds 1000*cfg+batch",
+                       "parallelism": "replicas only (no exchange step)" if world > 1 else "1 GPU",
+                       "launch": "back-to-back C-ABI calls on one stream"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "achieved": per_launch_gbs, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": per_launch_gbs / peaks["hbm_gbs"],
+                         "peak_kind": peak_kind, "frac_of_nominal_8TBs": per_launch_gbs / NOMINAL_HBM_GBS,
+                         "traffic": traffic.get(cfg.name), "kernel": "skinny_kernel<1,8>"},
+            "graph_replay_us_per_call": graph_us,
+            "cpu_baseline": cpu,
+            "configs": extra,
+        }
+        gemm = [r for r in extra if r["path"] == "tcgen05" and r["name"].startswith(("cfg4", "cfg5"))]
+        if gemm:
+            best = max(gemm, key=lambda r: r["TFLOPs"])
+            line["roofline_gemm"] = {"bound": "tensor", "achieved": best["TFLOPs"], "peak": peaks["bf16_tflops"],
+                                     "unit": "TFLOP/s", "frac": best["TFLOPs"] / peaks["bf16_tflops"],
+                                     "peak_kind": peak_kind + " (cuBLAS burst)", "workload": best["name"],
+                                     "traffic": traffic.get(best["name"]), "kernel": "gemm_tcgen05"}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--configs", default="1,3,4,5",
+                    help="1-based extra configs to time at --gpus 1 ('' for none)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    args.steps = max(args.steps, 1)
+    args.configs = [int(x) - 1 for x in args.configs.split(",") if x.strip()]
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,148 @@
+/*
+ * morello.h -- C ABI of the B200 (sm_100a) MatmulAccum library.
+ *
+ * The operation is the paper's accumulating batched matrix multiply
+ * (Section 2, "Tiling": dimensions are ordered batch, m, k, n and the output
+ * is shaped batch x m x n; Section 2.2: MatmulAccum is the accumulating member
+ * of the Matmul / MatmulAccum pair and its operands are typed bf16, bf16 and
+ * f32; a bf16 -> f32 Move is an exact upcast):
+ *
+ *     C[b,i,j]  <-  C[b,i,j] + sum_{p<k} A[b,i,p] * B[b,p,j]
+ *
+ * Layout (all entry points): dense row-major, no leading dimensions,
+ *     A[b][m][k]  bf16   (read only)
+ *     B[b][k][n]  bf16   (read only, one matrix per batch, no broadcasting)
+ *     C[b][m][n]  f32    (read-modify-write)
+ * Products are exact in f32; sums are accumulated in f32 (on the FP32 units or
+ * in the tensor cores' f32 accumulators) in an order that is fixed for a given
+ * shape and device, so repeated calls give identical bits.  C is added once,
+ * after the sum over k is complete.
+ *
+ * Ownership: the caller owns every buffer; the library keeps no reference to
+ * them after the enqueued work has run.  C must not overlap A, B or the
+ * workspace (not checked).  Unless stated otherwise pointers are DEVICE
+ * pointers on the current CUDA device, calls are asynchronous on `stream`
+ * (a cudaStream_t passed as void*; NULL is the legacy default stream) and
+ * never synchronise the host.
+ *
+ * Errors: the int return value (a morello_status_t) is the only channel.  On
+ * any error nothing is enqueued.  There is no CPU fallback: a device that is
+ * not compute capability 10.x yields MORELLO_ERR_UNSUPPORTED_DEVICE.
+ */
+#ifndef MORELLO_H_
+#define MORELLO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MORELLO_OK = 0,
+  MORELLO_ERR_INVALID_SHAPE = 1,      /* a dimension < 0, or a byte size overflows int64 */
+  MORELLO_ERR_NULL_POINTER = 2,       /* A, B or C null while its element count is > 0 */
+  MORELLO_ERR_MISALIGNED = 3,         /* A or B not 2-byte aligned, C not 4-byte aligned,
+                                         workspace not 16-byte aligned */
+  MORELLO_ERR_UNSUPPORTED_DEVICE = 4, /* current device is not compute capability 10.x */
+  MORELLO_ERR_WORKSPACE = 5,          /* workspace too small, or its allocation failed */
+  MORELLO_ERR_CUDA = 6,               /* a CUDA call failed; see morello_last_cuda_error() */
+  MORELLO_ERR_DEVICE_TIMEOUT = 7,     /* a bounded device-side wait gave up; only reported by
+                                         morello_read_device_status() */
+  MORELLO_ERR_UNSUPPORTED_PATH = 8    /* a forced path cannot run this shape / alignment */
+} morello_status_t;
+
+/* Kernel families behind the shape selector (Section 2 of the paper tiles one
+ * MatmulAccum into smaller ones; here the tiling is fixed per family). */
+enum {
+  MORELLO_PATH_AUTO = -1,
+  MORELLO_PATH_SKINNY = 0,  /* HBM-streaming FP32-FMA kernel, rows in chunks of <= 16 */
+  MORELLO_PATH_TCGEN05 = 1  /* TMA + tcgen05 tensor-core GEMM with fused C += epilogue */
+};
+
+/*
+ * MatmulAccum(b x m x k x n), the definition at the top of this file.
+ * Any dimension may be 0: b*m*n == 0 or k == 0 returns MORELLO_OK with C
+ * untouched (empty sum).  Scratch memory, when the chosen kernel needs any, is
+ * a per-device buffer owned by the library that grows on demand (the only
+ * allocation this call can make); concurrent calls on different streams that
+ * both need scratch must use morello_matmul_accum_ws instead.
+ */
+int morello_matmul_accum(int64_t b, int64_t m, int64_t k, int64_t n,
+                         const void* A, const void* B, float* C, void* stream);
+
+/*
+ * Bytes of scratch morello_matmul_accum_ws needs for this shape on the current
+ * device (0 if none; also 0 for invalid shapes).  The figure assumes A, B and
+ * C are 16-byte aligned; it is an upper bound otherwise.
+ */
+size_t morello_workspace_bytes(int64_t b, int64_t m, int64_t k, int64_t n);
+
+/*
+ * Same operation with caller-provided scratch: `workspace` is a device buffer
+ * of `workspace_bytes` >= morello_workspace_bytes(...), 16-byte aligned (may be
+ * NULL when 0 bytes are needed).  Its contents need no initialisation and are
+ * unspecified afterwards.  Makes no allocation.
+ */
+int morello_matmul_accum_ws(int64_t b, int64_t m, int64_t k, int64_t n,
+                            const void* A, const void* B, float* C,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * End-to-end convenience call on HOST buffers (same layouts): copies A, B and
+ * C to library-owned device staging (grown on demand), runs the operation,
+ * copies C back and synchronises before returning.  Pinned host memory makes
+ * the copies asynchronous with respect to each other but the call still
+ * returns only when C_host holds the result.
+ */
+int morello_matmul_accum_host(int64_t b, int64_t m, int64_t k, int64_t n,
+                              const void* A_host, const void* B_host, float* C_host);
+
+/* --- introspection and experiments (tests and benchmarks) ------------------ */
+
+/* The path the selector picks for this shape with 16-byte-aligned operands:
+ * MORELLO_PATH_SKINNY or MORELLO_PATH_TCGEN05 (-1 for an invalid shape). */
+int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n);
+
+/*
+ * Run on a given path (MORELLO_PATH_AUTO = selector) with a given split of the
+ * k range across thread blocks (0 = automatic).  Returns
+ * MORELLO_ERR_UNSUPPORTED_PATH, and enqueues nothing, when the path cannot run
+ * the shape (the tcgen05 path needs k % 8 == 0, n % 8 == 0 and 16-byte-aligned
+ * A, B, C).  workspace may be NULL with workspace_bytes 0 to use the library's
+ * own per-device scratch.
+ */
+int morello_matmul_accum_forced(int path, int split_k,
+                                int64_t b, int64_t m, int64_t k, int64_t n,
+                                const void* A, const void* B, float* C,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of scratch the forced variant needs for this path and split. */
+size_t morello_workspace_bytes_forced(int path, int split_k,
+                                      int64_t b, int64_t m, int64_t k, int64_t n);
+
+/*
+ * Synchronises `stream`, then reads and clears the device-side status word
+ * that bounded waits inside the kernels write when they give up.  Returns
+ * MORELLO_OK, MORELLO_ERR_DEVICE_TIMEOUT or MORELLO_ERR_CUDA.  If `detail` is
+ * not NULL it receives the raw status word (0 when OK).
+ */
+int morello_read_device_status(void* stream, uint32_t* detail);
+
+/* Kernel launches enqueued by this library since it was loaded (all devices). */
+uint64_t morello_launch_count(void);
+
+/* The cudaError_t of the most recent failed CUDA call on this thread (0 if none). */
+int morello_last_cuda_error(void);
+
+/* Static, NUL-terminated description of a status code. */
+const char* morello_status_string(int status);
+
+/* Static version string. */
+const char* morello_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MORELLO_H_ */

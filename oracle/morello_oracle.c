@@ -63,53 +63,61 @@ void oracle_matmul_accum_naive(int64_t b, int64_t m, int64_t k, int64_t n,
             }
 }
 
+/* Columns are handed out in blocks of this many, so that a problem with few
+ * rows (the vector-matrix multiply has one) still uses every host thread. */
+#define ORACLE_COL_BLOCK 1024
+
 /*
- * One output row (bb, i), all n columns: the same arithmetic per element in
- * the same p order as the triple loop, with the j loop innermost so that B is
- * walked along its rows.  `s` is a caller-provided buffer of n doubles.
- * If T is not NULL it receives sum_p |A[b,i,p] * B[b,p,j]| (the scale of the
- * floating-point tolerance) for the row.
+ * Columns [j0, j1) of one output row (bb, i): the same arithmetic per element
+ * in the same p order as the triple loop, with the j loop innermost so that B
+ * is walked along its rows.  `s` is a caller-provided buffer of j1 - j0
+ * doubles.  If T_row is not NULL it receives sum_p |A[b,i,p] * B[b,p,j]| (the
+ * scale of the floating-point tolerance) for those columns.
  */
 static void oracle_row(int64_t bb, int64_t i, int64_t m, int64_t k, int64_t n,
+                       int64_t j0, int64_t j1,
                        const uint16_t *A, const uint16_t *B,
                        const float *Cin_row, float *Cout_row, double *T_row,
                        double *s)
 {
-    for (int64_t j = 0; j < n; ++j) s[j] = (double)Cin_row[j];
-    if (T_row) for (int64_t j = 0; j < n; ++j) T_row[j] = 0.0;
+    for (int64_t j = j0; j < j1; ++j) s[j - j0] = (double)Cin_row[j];
+    if (T_row) for (int64_t j = j0; j < j1; ++j) T_row[j] = 0.0;
     for (int64_t p = 0; p < k; ++p) {
         const double a = bf16_to_double(A[(bb * m + i) * k + p]);
         const uint16_t *Brow = B + (bb * k + p) * n;
-        for (int64_t j = 0; j < n; ++j) s[j] += a * bf16_to_double(Brow[j]);
+        for (int64_t j = j0; j < j1; ++j) s[j - j0] += a * bf16_to_double(Brow[j]);
         if (T_row)
-            for (int64_t j = 0; j < n; ++j)
+            for (int64_t j = j0; j < j1; ++j)
                 T_row[j] += fabs(a * bf16_to_double(Brow[j]));
     }
-    for (int64_t j = 0; j < n; ++j) Cout_row[j] = (float)s[j];
+    for (int64_t j = j0; j < j1; ++j) Cout_row[j] = (float)s[j - j0];
 }
 
 /*
- * Whole problem, in place on C.  Rows (b, i) are independent, so they are
- * handed to host threads (OpenMP) when the library is built with -fopenmp;
- * the arithmetic of every element is unchanged by the threading.
- * Returns 0, or -1 if the scratch row could not be allocated.
+ * Whole problem, in place on C.  Output elements are independent, so (row,
+ * column block) tasks are handed to host threads (OpenMP) when the library is
+ * built with -fopenmp; the arithmetic of every element is unchanged by the
+ * threading.  Returns 0, or -1 if the scratch buffer could not be allocated.
  */
 int oracle_matmul_accum(int64_t b, int64_t m, int64_t k, int64_t n,
                         const uint16_t *A, const uint16_t *B, float *C)
 {
     if (b <= 0 || m <= 0 || n <= 0) return 0;
+    const int64_t nblk = (n + ORACLE_COL_BLOCK - 1) / ORACLE_COL_BLOCK;
     int failed = 0;
 #pragma omp parallel
     {
-        double *s = (double *)malloc((size_t)n * sizeof(double));
+        double *s = (double *)malloc(ORACLE_COL_BLOCK * sizeof(double));
         if (!s) {
 #pragma omp atomic write
             failed = 1;
         } else {
 #pragma omp for schedule(dynamic, 1)
-            for (int64_t r = 0; r < b * m; ++r) {
+            for (int64_t t = 0; t < b * m * nblk; ++t) {
+                const int64_t r = t / nblk, j0 = (t % nblk) * ORACLE_COL_BLOCK;
+                const int64_t j1 = j0 + ORACLE_COL_BLOCK < n ? j0 + ORACLE_COL_BLOCK : n;
                 float *row = C + r * n;
-                oracle_row(r / m, r % m, m, k, n, A, B, row, row, NULL, s);
+                oracle_row(r / m, r % m, m, k, n, j0, j1, A, B, row, row, NULL, s);
             }
         }
         free(s);
@@ -129,20 +137,23 @@ int oracle_matmul_accum_rows(int64_t b, int64_t m, int64_t k, int64_t n,
                              const int64_t *rows, float *out, double *T)
 {
     if (n <= 0 || nrows <= 0) return 0;
+    const int64_t nblk = (n + ORACLE_COL_BLOCK - 1) / ORACLE_COL_BLOCK;
     int failed = 0;
 #pragma omp parallel
     {
-        double *s = (double *)malloc((size_t)n * sizeof(double));
+        double *s = (double *)malloc(ORACLE_COL_BLOCK * sizeof(double));
         if (!s) {
 #pragma omp atomic write
             failed = 1;
         } else {
 #pragma omp for schedule(dynamic, 1)
-            for (int64_t t = 0; t < nrows; ++t) {
-                const int64_t r = rows[t];
+            for (int64_t t = 0; t < nrows * nblk; ++t) {
+                const int64_t q = t / nblk, j0 = (t % nblk) * ORACLE_COL_BLOCK;
+                const int64_t j1 = j0 + ORACLE_COL_BLOCK < n ? j0 + ORACLE_COL_BLOCK : n;
+                const int64_t r = rows[q];
                 if (r < 0 || r >= b * m) continue;
-                oracle_row(r / m, r % m, m, k, n, A, B, C_in + r * n,
-                           out + t * n, T ? T + t * n : NULL, s);
+                oracle_row(r / m, r % m, m, k, n, j0, j1, A, B, C_in + r * n,
+                           out + q * n, T ? T + q * n : NULL, s);
             }
         }
         free(s);

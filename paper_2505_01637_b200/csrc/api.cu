@@ -1,0 +1,334 @@
+// C ABI of the library: argument validation, per-device state, the shape
+// selector and the dispatch to the two kernel families.
+#include <algorithm>
+#include <atomic>
+#include <mutex>
+
+#include "../../include/morello.h"
+#include "internal.h"
+
+namespace morello {
+namespace {
+
+constexpr int kMaxDevices = 64;
+constexpr int kSkinnyMaxRows = 16;
+
+struct DeviceState {
+  bool ready = false;
+  int status_code = MORELLO_OK;  // result of the one-time set-up
+  DeviceInfo info;
+  void* scratch = nullptr;       // library-owned workspace, grown on demand
+  size_t scratch_bytes = 0;
+  void* stage = nullptr;         // device staging for the host-buffer entry point
+  size_t stage_bytes = 0;
+};
+
+std::mutex g_mutex;
+DeviceState g_dev[kMaxDevices];
+std::atomic<uint64_t> g_launches{0};
+thread_local int t_last_cuda_error = 0;
+
+int cuda_fail(cudaError_t e) {
+  t_last_cuda_error = (int)e;
+  (void)cudaGetLastError();
+  return MORELLO_ERR_CUDA;
+}
+
+// One-time set-up per device, under g_mutex.
+int device_state(DeviceState** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= kMaxDevices) return MORELLO_ERR_UNSUPPORTED_DEVICE;
+  DeviceState& st = g_dev[dev];
+  if (!st.ready) {
+    int major = 0, sms = 0;
+    if ((e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess)
+      return cuda_fail(e);
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+      return cuda_fail(e);
+    st.info.cc_major = major;
+    st.info.sms = sms;
+    if (major != 10) {
+      st.status_code = MORELLO_ERR_UNSUPPORTED_DEVICE;
+    } else {
+      if ((e = cudaMalloc((void**)&st.info.status, 256)) != cudaSuccess) return cuda_fail(e);
+      if ((e = cudaMemset(st.info.status, 0, 256)) != cudaSuccess) return cuda_fail(e);
+      st.status_code = MORELLO_OK;
+    }
+    st.ready = true;
+  }
+  *out = &st;
+  return st.status_code;
+}
+
+bool mul_overflows(int64_t a, int64_t b, int64_t* out) {
+  return __builtin_mul_overflow(a, b, out);
+}
+
+// Shape and pointer checks common to every entry point.  Sets *empty when there
+// is nothing to do.
+int validate(int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const void* B,
+             const void* C, bool* empty) {
+  *empty = false;
+  if (b < 0 || m < 0 || k < 0 || n < 0) return MORELLO_ERR_INVALID_SHAPE;
+  int64_t mk, kn, mn, t;
+  if (mul_overflows(m, k, &mk) || mul_overflows(k, n, &kn) || mul_overflows(m, n, &mn) ||
+      mul_overflows(b, mk, &t) || mul_overflows(t, 2, &t) || mul_overflows(b, kn, &t) ||
+      mul_overflows(t, 2, &t) || mul_overflows(b, mn, &t) || mul_overflows(t, 4 * 64, &t))
+    return MORELLO_ERR_INVALID_SHAPE;
+  if (b == 0 || m == 0 || n == 0 || k == 0) {
+    *empty = true;
+    return MORELLO_OK;
+  }
+  if (!A || !B || !C) return MORELLO_ERR_NULL_POINTER;
+  if (reinterpret_cast<uintptr_t>(A) % 2 || reinterpret_cast<uintptr_t>(B) % 2 ||
+      reinterpret_cast<uintptr_t>(C) % 4)
+    return MORELLO_ERR_MISALIGNED;
+  return MORELLO_OK;
+}
+
+int select_path(int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const void* B,
+                const void* C) {
+  if (m <= kSkinnyMaxRows) return MORELLO_PATH_SKINNY;
+  return gemm_shape_supported(b, m, k, n, A, B, C) ? MORELLO_PATH_TCGEN05 : MORELLO_PATH_SKINNY;
+}
+
+// Scratch for the skinny path over all row chunks (chunks run one after another on
+// the stream, so they share the buffer).
+size_t skinny_workspace(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int vec, int split_k) {
+  // Chunks are full (16 rows) except possibly the last one.
+  const int first = (int)std::min<int64_t>(kSkinnyMaxRows, m);
+  size_t need = skinny_plan(sms, b, first, k, n, vec, split_k).workspace_bytes;
+  const int last = (int)(m % kSkinnyMaxRows);
+  if (m > kSkinnyMaxRows && last != 0)
+    need = std::max(need, skinny_plan(sms, b, last, k, n, vec, split_k).workspace_bytes);
+  return need;
+}
+
+size_t workspace_for(int sms, int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n,
+                     int vec) {
+  if (path == MORELLO_PATH_TCGEN05) return gemm_plan(sms, b, m, k, n, split_k).workspace_bytes;
+  return skinny_workspace(sms, b, m, k, n, vec, split_k);
+}
+
+int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
+        const void* B, float* C, void* workspace, size_t workspace_bytes, bool own_scratch,
+        void* stream) {
+  bool empty = false;
+  int rc = validate(b, m, k, n, A, B, C, &empty);
+  if (rc != MORELLO_OK) return rc;
+  if (split_k < 0) return MORELLO_ERR_INVALID_SHAPE;
+  if (workspace && reinterpret_cast<uintptr_t>(workspace) % 16) return MORELLO_ERR_MISALIGNED;
+
+  DeviceState* st = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    rc = device_state(&st);
+  }
+  if (rc != MORELLO_OK) return rc;
+  if (empty) return MORELLO_OK;
+
+  if (path == MORELLO_PATH_AUTO) {
+    path = select_path(b, m, k, n, A, B, C);
+  } else if (path == MORELLO_PATH_TCGEN05) {
+    if (!gemm_shape_supported(b, m, k, n, A, B, C)) return MORELLO_ERR_UNSUPPORTED_PATH;
+  } else if (path != MORELLO_PATH_SKINNY) {
+    return MORELLO_ERR_UNSUPPORTED_PATH;
+  }
+
+  const int sms = st->info.sms;
+  const int vec = skinny_vec(n, B);
+  const size_t need = workspace_for(sms, path, split_k, b, m, k, n, vec);
+  float* ws = static_cast<float*>(workspace);
+  if (need > 0) {
+    if (own_scratch) {
+      std::lock_guard<std::mutex> lock(g_mutex);
+      if (st->scratch_bytes < need) {
+        // Work already enqueued may still be using the old buffer.
+        cudaError_t e = cudaDeviceSynchronize();
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (st->scratch) cudaFree(st->scratch);
+        st->scratch = nullptr;
+        st->scratch_bytes = 0;
+        const size_t grow = std::max(need, (size_t)(8u << 20));
+        if ((e = cudaMalloc(&st->scratch, grow)) != cudaSuccess) {
+          cuda_fail(e);
+          return MORELLO_ERR_WORKSPACE;
+        }
+        st->scratch_bytes = grow;
+      }
+      ws = static_cast<float*>(st->scratch);
+    } else if (!ws || workspace_bytes < need) {
+      return MORELLO_ERR_WORKSPACE;
+    }
+  }
+
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint64_t launches = 0;
+  cudaError_t e = cudaSuccess;
+  if (path == MORELLO_PATH_TCGEN05) {
+    const GemmPlan plan = gemm_plan(sms, b, m, k, n, split_k);
+    e = gemm_launch(st->info, plan, b, m, k, n, static_cast<const uint16_t*>(A),
+                    static_cast<const uint16_t*>(B), C, ws, s, &launches);
+  } else {
+    const uint16_t* a = static_cast<const uint16_t*>(A);
+    for (int64_t i0 = 0; i0 < m && e == cudaSuccess; i0 += kSkinnyMaxRows) {
+      const int mc = (int)std::min<int64_t>(kSkinnyMaxRows, m - i0);
+      const SkinnyPlan plan = skinny_plan(sms, b, mc, k, n, vec, split_k);
+      e = skinny_launch(plan, b, mc, k, n, a + i0 * k, m * k, static_cast<const uint16_t*>(B),
+                        C + i0 * n, m * n, ws, s, &launches);
+    }
+  }
+  g_launches.fetch_add(launches, std::memory_order_relaxed);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return MORELLO_OK;
+}
+
+}  // namespace
+}  // namespace morello
+
+using namespace morello;
+
+#pragma GCC visibility push(default)
+extern "C" {
+
+int morello_matmul_accum(int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
+                         const void* B, float* C, void* stream) {
+  return run(MORELLO_PATH_AUTO, 0, b, m, k, n, A, B, C, nullptr, 0, true, stream);
+}
+
+size_t morello_workspace_bytes(int64_t b, int64_t m, int64_t k, int64_t n) {
+  return morello_workspace_bytes_forced(MORELLO_PATH_AUTO, 0, b, m, k, n);
+}
+
+size_t morello_workspace_bytes_forced(int path, int split_k, int64_t b, int64_t m, int64_t k,
+                                      int64_t n) {
+  bool empty = false;
+  // A 16-byte-aligned stand-in address: only its alignment is looked at.
+  const void* fake = reinterpret_cast<const void*>(uintptr_t(4096));
+  if (validate(b, m, k, n, fake, fake, fake, &empty) != MORELLO_OK || empty || split_k < 0) return 0;
+  DeviceState* st = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (device_state(&st) != MORELLO_OK) return 0;
+  }
+  if (path == MORELLO_PATH_AUTO) path = select_path(b, m, k, n, fake, fake, fake);
+  if (path == MORELLO_PATH_TCGEN05 && !gemm_shape_supported(b, m, k, n, fake, fake, fake)) return 0;
+  return workspace_for(st->info.sms, path, split_k, b, m, k, n, skinny_vec(n, fake));
+}
+
+int morello_matmul_accum_ws(int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
+                            const void* B, float* C, void* workspace, size_t workspace_bytes,
+                            void* stream) {
+  return run(MORELLO_PATH_AUTO, 0, b, m, k, n, A, B, C, workspace, workspace_bytes, false, stream);
+}
+
+int morello_matmul_accum_forced(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n,
+                                const void* A, const void* B, float* C, void* workspace,
+                                size_t workspace_bytes, void* stream) {
+  const bool own = (workspace == nullptr && workspace_bytes == 0);
+  return run(path, split_k, b, m, k, n, A, B, C, workspace, workspace_bytes, own, stream);
+}
+
+int morello_matmul_accum_host(int64_t b, int64_t m, int64_t k, int64_t n, const void* A_host,
+                              const void* B_host, float* C_host) {
+  bool empty = false;
+  int rc = validate(b, m, k, n, A_host, B_host, C_host, &empty);
+  if (rc != MORELLO_OK) return rc;
+  DeviceState* st = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    rc = device_state(&st);
+  }
+  if (rc != MORELLO_OK || empty) return rc;
+  auto round256 = [](size_t x) { return (x + 255) / 256 * 256; };
+  const size_t a_bytes = (size_t)b * m * k * 2, b_bytes = (size_t)b * k * n * 2,
+               c_bytes = (size_t)b * m * n * 4;
+  const size_t need = round256(a_bytes) + round256(b_bytes) + round256(c_bytes);
+  cudaError_t e;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (st->stage_bytes < need) {
+      if ((e = cudaDeviceSynchronize()) != cudaSuccess) return cuda_fail(e);
+      if (st->stage) cudaFree(st->stage);
+      st->stage = nullptr;
+      st->stage_bytes = 0;
+      if ((e = cudaMalloc(&st->stage, need)) != cudaSuccess) {
+        cuda_fail(e);
+        return MORELLO_ERR_WORKSPACE;
+      }
+      st->stage_bytes = need;
+    }
+  }
+  char* base = static_cast<char*>(st->stage);
+  void* dA = base;
+  void* dB = base + round256(a_bytes);
+  float* dC = reinterpret_cast<float*>(base + round256(a_bytes) + round256(b_bytes));
+  cudaStream_t s = cudaStreamPerThread;
+  if ((e = cudaMemcpyAsync(dA, A_host, a_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(dC, C_host, c_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+    return cuda_fail(e);
+  rc = run(MORELLO_PATH_AUTO, 0, b, m, k, n, dA, dB, dC, nullptr, 0, true, s);
+  if (rc != MORELLO_OK) {
+    cudaStreamSynchronize(s);
+    return rc;
+  }
+  if ((e = cudaMemcpyAsync(C_host, dC, c_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess ||
+      (e = cudaStreamSynchronize(s)) != cudaSuccess)
+    return cuda_fail(e);
+  return MORELLO_OK;
+}
+
+int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n) {
+  bool empty = false;
+  const void* fake = reinterpret_cast<const void*>(uintptr_t(4096));
+  if (validate(b, m, k, n, fake, fake, fake, &empty) != MORELLO_OK) return -1;
+  return select_path(b, m, k, n, fake, fake, fake);
+}
+
+int morello_read_device_status(void* stream, uint32_t* detail) {
+  if (detail) *detail = 0;
+  DeviceState* st = nullptr;
+  int rc;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    rc = device_state(&st);
+  }
+  if (rc != MORELLO_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return cuda_fail(e);
+  uint32_t word = 0;
+  if ((e = cudaMemcpy(&word, st->info.status, 4, cudaMemcpyDeviceToHost)) != cudaSuccess)
+    return cuda_fail(e);
+  if (word == 0) return MORELLO_OK;
+  if ((e = cudaMemset(st->info.status, 0, 4)) != cudaSuccess) return cuda_fail(e);
+  if (detail) *detail = word;
+  return MORELLO_ERR_DEVICE_TIMEOUT;
+}
+
+uint64_t morello_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int morello_last_cuda_error(void) { return t_last_cuda_error; }
+
+const char* morello_status_string(int status) {
+  switch (status) {
+    case MORELLO_OK: return "ok";
+    case MORELLO_ERR_INVALID_SHAPE: return "invalid shape (negative dimension or size overflow)";
+    case MORELLO_ERR_NULL_POINTER: return "null pointer for a non-empty tensor";
+    case MORELLO_ERR_MISALIGNED: return "pointer not aligned to its element type (or workspace to 16 bytes)";
+    case MORELLO_ERR_UNSUPPORTED_DEVICE: return "current device is not compute capability 10.x";
+    case MORELLO_ERR_WORKSPACE: return "workspace too small or its allocation failed";
+    case MORELLO_ERR_CUDA: return "a CUDA call failed (see morello_last_cuda_error)";
+    case MORELLO_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
+    case MORELLO_ERR_UNSUPPORTED_PATH: return "the forced path cannot run this shape or alignment";
+    default: return "unknown status";
+  }
+}
+
+const char* morello_version(void) { return "morello-b200 0.1 (sm_100a)"; }
+
+}  // extern "C"
+#pragma GCC visibility pop

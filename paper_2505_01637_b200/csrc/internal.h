@@ -1,0 +1,61 @@
+// Internal declarations shared by the translation units of the CUDA library.
+// Nothing here is visible through the C ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace morello {
+
+// Device-side status word written by bounded waits that gave up.
+// 0 = OK; otherwise (site << 16) | detail, first writer wins.
+struct DeviceInfo {
+  int sms = 0;
+  int cc_major = 0;
+  uint32_t* status = nullptr;  // one zero-initialised word in device memory
+};
+
+// ---- skinny path (FP32 FMA, rows in chunks of <= 16) -------------------------
+struct SkinnyPlan {
+  int m_tile;        // 1, 2, 4, 8 or 16: compile-time row count of the kernel used
+  int vec;           // bf16 elements per load: 8, 4, 2 or 1
+  int units;         // column units (of `vec` columns) per thread block
+  int row_lanes;     // k rows visited per pass of a thread block
+  int threads;       // launch width (multiple of 32, >= units * row_lanes)
+  int col_blocks;    // thread blocks along n
+  int split_k;       // thread blocks along k
+  int64_t k_per_split;
+  int k_chunk;       // k rows of A staged in shared memory at a time
+  size_t smem_bytes;
+  size_t workspace_bytes;  // partial sums [split_k][b][m][n] f32 when split_k > 1
+};
+
+// Chooses the decomposition for rows [0, m) with m <= 16.  split_k 0 = automatic.
+SkinnyPlan skinny_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int vec, int split_k);
+
+// Largest vector width (in bf16 elements) the operands' alignment and n allow.
+int skinny_vec(int64_t n, const void* B);
+
+// Enqueues C[:, i0:i0+m, :] += A[:, i0:i0+m, :] x B for m <= 16 (one row chunk).
+// a_batch / c_batch are the batch strides in elements of the full tensors.
+cudaError_t skinny_launch(const SkinnyPlan& plan, int64_t b, int m, int64_t k, int64_t n,
+                          const uint16_t* A, int64_t a_batch, const uint16_t* B, float* C,
+                          int64_t c_batch, float* workspace, cudaStream_t stream,
+                          uint64_t* launches);
+
+// ---- tcgen05 path ------------------------------------------------------------
+struct GemmPlan {
+  bool supported;
+  int split_k;
+  size_t workspace_bytes;
+};
+
+bool gemm_shape_supported(int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
+                          const void* B, const void* C);
+GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int split_k);
+cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m,
+                        int64_t k, int64_t n, const uint16_t* A, const uint16_t* B, float* C,
+                        float* workspace, cudaStream_t stream, uint64_t* launches);
+
+}  // namespace morello

@@ -1,0 +1,350 @@
+// Skinny MatmulAccum: C[b, 0:m, :] += A[b, 0:m, :] x B[b] for m <= 16 on the
+// FP32 FMA units, streaming B from HBM exactly once.
+//
+// Decomposition.  The n columns are cut into "units" of VEC columns (one
+// 2*VEC-byte load).  A thread block owns `units` adjacent units and one slice
+// of the k range; its threads form a (row_lanes x units) grid: thread
+// (r, u) visits rows r, r + row_lanes, ... of the slice and keeps M x VEC f32
+// accumulators for unit u.  A warp therefore reads contiguous 2*VEC*units-byte
+// row segments, and every thread has UNROLL independent loads in flight.
+// The rows of A that the slice needs sit in shared memory as f32, transposed to
+// [k][M] so that one thread reads its M multipliers with vector loads.
+// At the end the row lanes are summed through shared memory in a fixed order
+// (lane 0, 1, 2, ...), so results are deterministic.  With one k slice the
+// block adds its sums to C itself; with several it writes them to
+// partial[slice][b][m][n] and reduce_kernel adds the slices in slice order and
+// then adds C once.
+#include <algorithm>
+
+#include "internal.h"
+
+namespace morello {
+namespace {
+
+constexpr int kSmemABudget = 64 * 1024;  // bytes of shared memory for the staged rows of A
+
+struct SkinnyParams {
+  const uint16_t* A;
+  const uint16_t* B;
+  float* C;
+  float* partial;
+  int64_t a_batch, b_batch, c_batch;  // batch strides in elements
+  int64_t k, n;
+  int64_t k_per_split;
+  int64_t partial_split_stride;  // b * m * n
+  int m;
+  int num_units;  // n / VEC
+  int units;
+  int row_lanes;
+  int col_blocks;
+  int split_k;
+  int k_chunk;
+};
+
+template <int M_T>
+struct Tuning;
+template <> struct Tuning<1>  { static constexpr int kThreads = 1024, kUnroll = 8; };
+template <> struct Tuning<2>  { static constexpr int kThreads = 1024, kUnroll = 8; };
+template <> struct Tuning<4>  { static constexpr int kThreads = 512,  kUnroll = 8; };
+template <> struct Tuning<8>  { static constexpr int kThreads = 512,  kUnroll = 4; };
+template <> struct Tuning<16> { static constexpr int kThreads = 256,  kUnroll = 4; };
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// Streaming loads of B: read-only path, no L1 allocation (every byte is used once).
+template <int VEC>
+struct BVec;
+template <> struct BVec<8> {
+  uint32_t w[4];
+  __device__ __forceinline__ void load(const uint16_t* p) {
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "l"(p));
+  }
+  __device__ __forceinline__ float get(int j) const { return (j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]); }
+};
+template <> struct BVec<4> {
+  uint32_t w[2];
+  __device__ __forceinline__ void load(const uint16_t* p) {
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];"
+                 : "=r"(w[0]), "=r"(w[1]) : "l"(p));
+  }
+  __device__ __forceinline__ float get(int j) const { return (j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]); }
+};
+template <> struct BVec<2> {
+  uint32_t w[1];
+  __device__ __forceinline__ void load(const uint16_t* p) {
+    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(w[0]) : "l"(p));
+  }
+  __device__ __forceinline__ float get(int j) const { return (j & 1) ? bf16_hi(w[0]) : bf16_lo(w[0]); }
+};
+template <> struct BVec<1> {
+  uint16_t h;
+  __device__ __forceinline__ void load(const uint16_t* p) {
+    asm volatile("ld.global.nc.L1::no_allocate.u16 %0, [%1];" : "=h"(h) : "l"(p));
+  }
+  __device__ __forceinline__ float get(int) const { return __uint_as_float(((uint32_t)h) << 16); }
+};
+
+template <int M_T, int VEC>
+__device__ __forceinline__ void fma_row(float (&acc)[M_T][VEC], const float* __restrict__ a_row,
+                                        const BVec<VEC>& v) {
+  float a[M_T];
+  if constexpr (M_T >= 4) {
+#pragma unroll
+    for (int i = 0; i < M_T; i += 4) {
+      const float4 q = *reinterpret_cast<const float4*>(a_row + i);
+      a[i] = q.x; a[i + 1] = q.y; a[i + 2] = q.z; a[i + 3] = q.w;
+    }
+  } else if constexpr (M_T == 2) {
+    const float2 q = *reinterpret_cast<const float2*>(a_row);
+    a[0] = q.x; a[1] = q.y;
+  } else {
+    a[0] = a_row[0];
+  }
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) {
+    const float bj = v.get(j);
+#pragma unroll
+    for (int i = 0; i < M_T; ++i) acc[i][j] = fmaf(a[i], bj, acc[i][j]);
+  }
+}
+
+template <int M_T, int VEC>
+__global__ void __launch_bounds__(Tuning<M_T>::kThreads)
+skinny_kernel(const SkinnyParams p) {
+  constexpr int UNROLL = Tuning<M_T>::kUnroll;
+  extern __shared__ __align__(16) float smem[];
+  float* a_s = smem;                                  // [k_chunk][M_T]
+  float* red = smem + (size_t)p.k_chunk * M_T;        // [row_lanes][M_T * units * VEC]
+
+  const int t = threadIdx.x;
+  const int ul = t % p.units;
+  const int rl = t / p.units;
+  const int cb = blockIdx.x % p.col_blocks;
+  const int s = blockIdx.x / p.col_blocks;
+  const int bb = blockIdx.y;
+  const int unit = cb * p.units + ul;
+  const bool active = (rl < p.row_lanes) && (unit < p.num_units);
+  const int64_t k0 = (int64_t)s * p.k_per_split;
+  const int64_t k1 = min(p.k, k0 + p.k_per_split);
+  const int R = p.row_lanes;
+
+  float acc[M_T][VEC];
+#pragma unroll
+  for (int i = 0; i < M_T; ++i)
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) acc[i][j] = 0.f;
+
+  const uint16_t* a_base = p.A + (int64_t)bb * p.a_batch;
+  const uint16_t* b_base = p.B + (int64_t)bb * p.b_batch + (int64_t)unit * VEC;
+
+  for (int64_t kc0 = k0; kc0 < k1; kc0 += p.k_chunk) {
+    const int kcl = (int)min((int64_t)p.k_chunk, k1 - kc0);
+    if (kc0 != k0) __syncthreads();  // previous chunk's readers are done with a_s
+#pragma unroll
+    for (int i = 0; i < M_T; ++i) {
+      for (int q = t; q < kcl; q += blockDim.x) {
+        const float v = (i < p.m)
+            ? __uint_as_float(((uint32_t)a_base[(int64_t)i * p.k + kc0 + q]) << 16) : 0.f;
+        a_s[q * M_T + i] = v;
+      }
+    }
+    __syncthreads();
+    if (active) {
+      const uint16_t* bp = b_base + (kc0 + rl) * p.n;
+      const int64_t step = (int64_t)R * p.n;
+      int q = rl;
+      for (; q + (UNROLL - 1) * R < kcl; q += UNROLL * R) {
+        BVec<VEC> v[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) v[u].load(bp + u * step);
+        bp += UNROLL * step;
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) fma_row<M_T, VEC>(acc, a_s + (q + u * R) * M_T, v[u]);
+      }
+      for (; q < kcl; q += R) {
+        BVec<VEC> v;
+        v.load(bp);
+        bp += step;
+        fma_row<M_T, VEC>(acc, a_s + q * M_T, v);
+      }
+    }
+  }
+
+  // Sum the row lanes in lane order through shared memory.
+  const int W = M_T * p.units * VEC;  // floats per row lane
+  if (active) {
+    float* dst = red + (size_t)rl * W + ul * VEC;
+#pragma unroll
+    for (int i = 0; i < M_T; ++i)
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) dst[i * p.units * VEC + j] = acc[i][j];
+  }
+  __syncthreads();
+  const int cols_here = p.units * VEC;
+  const int64_t col_base = (int64_t)cb * cols_here;
+  for (int o = t; o < W; o += blockDim.x) {
+    const int i = o / cols_here;
+    const int64_t col = col_base + (o - i * cols_here);
+    if (i >= p.m || col >= p.n) continue;
+    float sum = red[o];
+    for (int r = 1; r < R; ++r) sum += red[(size_t)r * W + o];
+    if (p.split_k == 1) {
+      float* c = p.C + (int64_t)bb * p.c_batch + (int64_t)i * p.n + col;
+      *c = *c + sum;
+    } else {
+      p.partial[(int64_t)s * p.partial_split_stride + ((int64_t)bb * p.m + i) * p.n + col] = sum;
+    }
+  }
+}
+
+// C[b, i, :] += sum over slices, slice order fixed; one thread per output element.
+__global__ void __launch_bounds__(256)
+reduce_kernel(const float* __restrict__ partial, float* __restrict__ C, int64_t total,
+              int64_t mn, int64_t c_batch, int split_k) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  float sum = partial[idx];
+  for (int s = 1; s < split_k; ++s) sum += partial[(int64_t)s * total + idx];
+  const int64_t bb = idx / mn;
+  float* c = C + bb * c_batch + (idx - bb * mn);
+  *c = *c + sum;
+}
+
+template <int M_T, int VEC>
+cudaError_t launch_one(const SkinnyPlan& plan, const SkinnyParams& prm, int64_t b,
+                       cudaStream_t stream) {
+  auto kern = skinny_kernel<M_T, VEC>;
+  if (plan.smem_bytes > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)plan.smem_bytes);
+    if (e != cudaSuccess) return e;
+  }
+  dim3 grid((unsigned)(plan.col_blocks * plan.split_k), (unsigned)b, 1);
+  kern<<<grid, plan.threads, plan.smem_bytes, stream>>>(prm);
+  return cudaGetLastError();
+}
+
+template <int M_T>
+cudaError_t launch_vec(const SkinnyPlan& plan, const SkinnyParams& prm, int64_t b,
+                       cudaStream_t stream) {
+  switch (plan.vec) {
+    case 8: return launch_one<M_T, 8>(plan, prm, b, stream);
+    case 4: return launch_one<M_T, 4>(plan, prm, b, stream);
+    case 2: return launch_one<M_T, 2>(plan, prm, b, stream);
+    default: return launch_one<M_T, 1>(plan, prm, b, stream);
+  }
+}
+
+int max_threads_for(int m_tile) {
+  switch (m_tile) {
+    case 1: return Tuning<1>::kThreads;
+    case 2: return Tuning<2>::kThreads;
+    case 4: return Tuning<4>::kThreads;
+    case 8: return Tuning<8>::kThreads;
+    default: return Tuning<16>::kThreads;
+  }
+}
+
+}  // namespace
+
+int skinny_vec(int64_t n, const void* B) {
+  const uintptr_t addr = reinterpret_cast<uintptr_t>(B);
+  for (int vec = 8; vec > 1; vec >>= 1)
+    if (n % vec == 0 && addr % (2 * vec) == 0) return vec;
+  return 1;
+}
+
+SkinnyPlan skinny_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int vec, int split_k) {
+  SkinnyPlan pl{};
+  pl.m_tile = m <= 1 ? 1 : m <= 2 ? 2 : m <= 4 ? 4 : m <= 8 ? 8 : 16;
+  pl.vec = vec;
+  const int max_threads = max_threads_for(pl.m_tile);
+  const int64_t num_units = n / vec;
+  const int unit_cap = (int)std::min<int64_t>(num_units, 128 / vec);  // <= 256-byte row segments
+  // One wave of thread blocks over the SMs when the columns allow it.
+  const int64_t per_sm = (b * num_units + sms - 1) / sms;
+  int units;
+  if (per_sm <= unit_cap) {
+    units = (int)std::max<int64_t>(per_sm, 1);
+  } else {
+    const int64_t waves = (per_sm + unit_cap - 1) / unit_cap;
+    units = (int)((per_sm + waves - 1) / waves);
+  }
+  units = std::min<int>(units, unit_cap);
+  pl.units = units;
+  pl.col_blocks = (int)((num_units + units - 1) / units);
+  const int64_t blocks = b * pl.col_blocks;
+  int s = split_k;
+  if (s <= 0) {
+    s = 1;
+    if (blocks * 2 <= sms && k >= 512)
+      s = (int)std::min<int64_t>(std::min<int64_t>(sms / blocks, k / 256), 32);
+  }
+  s = (int)std::max<int64_t>(1, std::min<int64_t>(s, std::max<int64_t>(k, 1)));
+  int64_t kps = (std::max<int64_t>(k, 1) + s - 1) / s;
+  kps = (kps + 7) / 8 * 8;
+  pl.k_per_split = kps;
+  pl.split_k = (int)((std::max<int64_t>(k, 1) + kps - 1) / kps);
+  // Row lanes: as many as the thread budget allows, a multiple of 8 when possible,
+  // never more than the slice has rows.
+  int rows = max_threads / units;
+  if (rows >= 8) rows = rows / 8 * 8;
+  rows = (int)std::max<int64_t>(1, std::min<int64_t>(rows, kps));
+  pl.row_lanes = rows;
+  pl.threads = (rows * units + 31) / 32 * 32;
+  pl.k_chunk = (int)std::min<int64_t>(kps, kSmemABudget / (4 * pl.m_tile));
+  pl.smem_bytes = (size_t)pl.k_chunk * pl.m_tile * 4 +
+                  (size_t)rows * pl.m_tile * units * vec * 4;
+  pl.workspace_bytes = pl.split_k > 1 ? (size_t)pl.split_k * b * m * n * 4 : 0;
+  return pl;
+}
+
+cudaError_t skinny_launch(const SkinnyPlan& plan, int64_t b, int m, int64_t k, int64_t n,
+                          const uint16_t* A, int64_t a_batch, const uint16_t* B, float* C,
+                          int64_t c_batch, float* workspace, cudaStream_t stream,
+                          uint64_t* launches) {
+  SkinnyParams prm{};
+  prm.A = A; prm.B = B; prm.C = C; prm.partial = workspace;
+  prm.a_batch = a_batch; prm.b_batch = k * n; prm.c_batch = c_batch;
+  prm.k = k; prm.n = n;
+  prm.k_per_split = plan.k_per_split;
+  prm.partial_split_stride = b * m * n;
+  prm.m = m;
+  prm.num_units = (int)(n / plan.vec);
+  prm.units = plan.units;
+  prm.row_lanes = plan.row_lanes;
+  prm.col_blocks = plan.col_blocks;
+  prm.split_k = plan.split_k;
+  prm.k_chunk = plan.k_chunk;
+  // grid.y carries the batch index; larger batches go in slabs.
+  for (int64_t b0 = 0; b0 < b; b0 += 65535) {
+    const int64_t bn = std::min<int64_t>(65535, b - b0);
+    SkinnyParams q = prm;
+    q.A = A + b0 * a_batch; q.B = B + b0 * k * n; q.C = C + b0 * c_batch;
+    q.partial = workspace ? workspace + b0 * m * n : nullptr;
+    cudaError_t e;
+    switch (plan.m_tile) {
+      case 1: e = launch_vec<1>(plan, q, bn, stream); break;
+      case 2: e = launch_vec<2>(plan, q, bn, stream); break;
+      case 4: e = launch_vec<4>(plan, q, bn, stream); break;
+      case 8: e = launch_vec<8>(plan, q, bn, stream); break;
+      default: e = launch_vec<16>(plan, q, bn, stream); break;
+    }
+    if (e != cudaSuccess) return e;
+    ++*launches;
+  }
+  if (plan.split_k > 1) {
+    const int64_t total = b * m * n;
+    const int64_t blocks = (total + 255) / 256;
+    reduce_kernel<<<(unsigned)blocks, 256, 0, stream>>>(workspace, C, total, (int64_t)m * n,
+                                                        c_batch, plan.split_k);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    ++*launches;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace morello

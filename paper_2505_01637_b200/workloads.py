@@ -145,12 +145,13 @@ def crc32(x: np.ndarray) -> int:
     return zlib.crc32(np.ascontiguousarray(x).view(np.uint8).reshape(-1).data) & 0xFFFFFFFF
 
 
-def sample_rows(b, m, seed, edge=128, per_batch=32):
-    """Flattened row ids (bb*m + i): the first and last ``edge`` rows of batch 0
-    plus ``per_batch`` seeded random rows of every batch (sorted, unique)."""
+def sample_rows(b, m, seed, edge=128, stride=64):
+    """Flattened row ids (bb*m + i) for sampled checks of a large problem: the
+    first and last ``edge`` rows of batch 0 plus, in every batch, one seeded
+    random row out of each block of ``stride`` rows (sorted, unique)."""
     rng = np.random.Generator(np.random.Philox(seed))
     rows = set(range(min(edge, m))) | set(range(max(0, m - edge), m))
     for beta in range(b):
-        for i in rng.integers(0, m, size=min(per_batch, m)):
-            rows.add(beta * m + int(i))
+        for i0 in range(0, m, stride):
+            rows.add(beta * m + i0 + int(rng.integers(0, min(stride, m - i0))))
     return np.array(sorted(rows), dtype=np.int64)
