@@ -13,8 +13,9 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmorello.so")
-SOURCES = ["api.cu", "skinny.cu", "gemm_tcgen05.cu"]
-HEADERS = [os.path.join(CSRC, "internal.h"),
+SOURCES = ["api.cu", "skinny.cu", "gemm_tcgen05.cu", "tensormap.cu"]
+HEADERS = [os.path.join(CSRC, "internal.h"), os.path.join(CSRC, "sm100.cuh"),
+           os.path.join(CSRC, "tensormap.h"),
            os.path.join(os.path.dirname(HERE), "include", "morello.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",

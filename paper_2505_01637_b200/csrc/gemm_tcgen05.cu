@@ -1,19 +1,328 @@
-// tcgen05 GEMM path (placeholder until the tensor-core kernel lands): reports every
-// shape as unsupported so that the selector keeps to the skinny path.
+// Tensor-core MatmulAccum for sm_100a: C[b] += A[b] x B[b] with bf16 operands and
+// f32 accumulation in tensor memory.
+//
+// One persistent thread block per SM walks 128 x 256 output tiles.  Its warps are
+// specialised:
+//   warp 0   producer: TMA loads of a 128 x 64 tile of A and a 64 x 256 tile of B per
+//            k block into a ring of shared-memory stages (128-byte swizzle);
+//   warp 1   MMA issuer: one elected lane issues tcgen05.mma (M 128, N 256, K 16), four
+//            per k block, accumulating in one of two 256-column TMEM buffers, and
+//            commits to the stage's "empty" barrier and, after the last k block, to the
+//            buffer's "full" barrier;
+//   warps 2-5 epilogue: read the accumulator with tcgen05.ld (each warp its own 32-lane
+//            quarter), add it to C in global memory (one rounding per element), and hand
+//            the buffer back.  The epilogue of tile i overlaps the main loop of tile i+1.
+// A is [m][k] (K-major operand).  B is [k][n], i.e. N is contiguous: it is fed as an
+// MN-major operand, each 64-column group of the tile being one TMA box of 64 k rows.
+// Rows, columns and k blocks past the tensor edge are zero-filled by TMA and the
+// epilogue predicates its accesses, so m, n and k need not be multiples of the tile.
+// Every barrier wait is bounded (sm100::mbar_wait); on a timeout the block stops
+// issuing work, records a status word and exits after releasing its TMEM.
+#include <algorithm>
+#include <mutex>
+
 #include "internal.h"
+#include "sm100.cuh"
+#include "tensormap.h"
 
 namespace morello {
+namespace {
 
-bool gemm_shape_supported(int64_t, int64_t, int64_t, int64_t, const void*, const void*,
-                          const void*) {
-  return false;
+using namespace sm100;
+
+constexpr int kTileM = 128;
+constexpr int kTileN = 256;
+constexpr int kTileK = 64;                         // one 128-byte swizzle span of bf16
+constexpr int kStages = 4;
+constexpr int kBytesA = kTileM * kTileK * 2;       // 16 KiB
+constexpr int kBytesB = kTileK * kTileN * 2;       // 32 KiB, as 4 boxes of 64 k x 64 n
+constexpr int kBoxBytesB = kTileK * 64 * 2;        // 8 KiB
+constexpr int kStageBytes = kBytesA + kBytesB;
+constexpr int kAccColumns = kTileN;                // f32 columns per accumulator buffer
+constexpr int kTmemColumns = 2 * kAccColumns;      // 512: the whole tensor memory
+constexpr int kThreads = 192;
+constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256;
+
+struct GemmParams {
+  float* C;
+  int64_t m, n, k;
+  int64_t c_batch;  // m * n
+  int m_tiles, n_tiles;
+  int64_t tiles;    // b * m_tiles * n_tiles
+  int k_blocks;
+  uint32_t* status;
+};
+
+struct Barriers {
+  uint64_t full[kStages];
+  uint64_t empty[kStages];
+  uint64_t acc_full[2];
+  uint64_t acc_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+            const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  // Stage buffers must sit on 1024-byte boundaries (the swizzle pattern repeats every
+  // 8 rows of 128 bytes and is keyed on address bits 7-9).
+  uint8_t* stages = reinterpret_cast<uint8_t*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  Barriers* bars = reinterpret_cast<Barriers*>(stages + (size_t)kStages * kStageBytes);
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&bars->full[s], 1);
+      mbar_init(&bars->empty[s], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bars->acc_full[i], 1);
+      mbar_init(&bars->acc_empty[i], 4);
+    }
+    bars->abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_descriptor(&map_a);
+    tma_prefetch_descriptor(&map_b);
+  }
+  if (warp == 1) {
+    tmem_alloc(&bars->tmem_base, kTmemColumns);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  // Everything above touched no global memory; from here on the predecessor on the
+  // stream must have completed.
+  pdl_wait();
+  pdl_release();
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (elect_one()) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int64_t t = blockIdx.x; t < p.tiles && ok; t += gridDim.x) {
+        const int mt = (int)(t % p.m_tiles);
+        const int nt = (int)((t / p.m_tiles) % p.n_tiles);
+        const int bb = (int)(t / ((int64_t)p.m_tiles * p.n_tiles));
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!(ok = mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag, p.status, 1))) break;
+          uint8_t* sa = stages + (size_t)stage * kStageBytes;
+          uint8_t* sb = sa + kBytesA;
+          mbar_arrive_expect_tx(&bars->full[stage], kStageBytes);
+          tma_load_3d(sa, &map_a, &bars->full[stage], kb * kTileK, mt * kTileM, bb);
+#pragma unroll
+          for (int j = 0; j < kTileN / 64; ++j)
+            tma_load_3d(sb + j * kBoxBytesB, &map_b, &bars->full[stage], nt * kTileN + j * 64,
+                        kb * kTileK, bb);
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (elect_one()) {
+      constexpr uint32_t idesc = instr_desc_bf16(kTileM, kTileN, false, true);
+      int stage = 0;
+      uint32_t phase = 0;
+      int buf = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int64_t t = blockIdx.x; t < p.tiles && ok; t += gridDim.x) {
+        if (!(ok = mbar_wait(&bars->acc_empty[buf], acc_phase ^ 1, abort_flag, p.status, 2))) break;
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + (uint32_t)buf * kAccColumns;
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!(ok = mbar_wait(&bars->full[stage], phase, abort_flag, p.status, 3))) break;
+          tc_fence_after_sync();
+          const uint32_t sa = smem_u32(stages + (size_t)stage * kStageBytes);
+          const uint32_t sb = sa + kBytesA;
+#pragma unroll
+          for (int j = 0; j < kTileK / 16; ++j) {
+            // A, K-major: 8-row groups 1024 bytes apart; 16 k elements = 32 bytes along the row.
+            const uint64_t da = smem_desc_sw128(sa + j * 32, 16, 1024);
+            // B, MN-major: 64-column groups one TMA box (8 KiB) apart, 8-row k groups 1024 bytes
+            // apart; 16 k rows = 2048 bytes.
+            const uint64_t db = smem_desc_sw128(sb + j * 2048, kBoxBytesB, 1024);
+            mma_bf16_ss(d_tmem, da, db, idesc, (kb | j) != 0 ? 1u : 0u);
+          }
+          mma_commit(&bars->empty[stage]);  // stage reusable once these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        mma_commit(&bars->acc_full[buf]);
+        if (++buf == 2) { buf = 0; acc_phase ^= 1; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int quarter = warp & 3;  // TMEM lanes [32 * quarter, 32 * quarter + 32)
+    int buf = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int64_t t = blockIdx.x; t < p.tiles && ok; t += gridDim.x) {
+      const int mt = (int)(t % p.m_tiles);
+      const int nt = (int)((t / p.m_tiles) % p.n_tiles);
+      const int64_t bb = t / ((int64_t)p.m_tiles * p.n_tiles);
+      ok = mbar_wait(&bars->acc_full[buf], acc_phase, abort_flag, p.status, 4);
+      ok = __all_sync(0xffffffffu, ok);  // also reconverges the warp for the aligned TMEM loads
+      if (!ok) break;
+      tc_fence_after_sync();
+      const int64_t row = (int64_t)mt * kTileM + quarter * 32 + lane;
+      const int64_t col0 = (int64_t)nt * kTileN;
+      float* crow = p.C + bb * p.c_batch + row * p.n + col0;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * kAccColumns;
+#pragma unroll 1
+      for (int c = 0; c < kTileN; c += 32) {
+        uint32_t r[32];
+        tmem_ld_32x32(taddr + c, r);
+        tmem_ld_wait();
+        if (row < p.m) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            if (col0 + c + j < p.n) {  // n is a multiple of 4 on this path
+              float4* dst = reinterpret_cast<float4*>(crow + c + j);
+              float4 v = *dst;
+              v.x += __uint_as_float(r[j]);
+              v.y += __uint_as_float(r[j + 1]);
+              v.z += __uint_as_float(r[j + 2]);
+              v.w += __uint_as_float(r[j + 3]);
+              *dst = v;
+            }
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->acc_empty[buf]);
+      if (++buf == 2) { buf = 0; acc_phase ^= 1; }
+    }
+  }
+
+  // Teardown: every role is done (or has given up); TMEM goes back before exit.
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc(tmem_base, kTmemColumns);
+  }
 }
 
-GemmPlan gemm_plan(int, int64_t, int64_t, int64_t, int64_t, int) { return GemmPlan{false, 1, 0}; }
+// Tensor maps are cached per (pointer, shape): encoding one costs a few microseconds.
+struct MapKey {
+  const void* a;
+  const void* b;
+  int64_t bsz, m, k, n;
+  bool operator==(const MapKey& o) const {
+    return a == o.a && b == o.b && bsz == o.bsz && m == o.m && k == o.k && n == o.n;
+  }
+};
+struct MapEntry {
+  MapKey key;
+  CUtensorMap map_a, map_b;
+  uint64_t stamp;
+  bool valid;
+};
+constexpr int kMapCache = 32;
+MapEntry g_maps[kMapCache];
+uint64_t g_stamp = 0;
+std::mutex g_map_mutex;
 
-cudaError_t gemm_launch(const DeviceInfo&, const GemmPlan&, int64_t, int64_t, int64_t, int64_t,
-                        const uint16_t*, const uint16_t*, float*, float*, cudaStream_t, uint64_t*) {
-  return cudaErrorNotSupported;
+cudaError_t get_maps(const MapKey& key, CUtensorMap* ma, CUtensorMap* mb) {
+  std::lock_guard<std::mutex> lock(g_map_mutex);
+  int victim = 0;   // an unused slot if there is one, else the least recently used
+  for (int i = 0; i < kMapCache; ++i) {
+    if (g_maps[i].valid && g_maps[i].key == key) {
+      g_maps[i].stamp = ++g_stamp;
+      *ma = g_maps[i].map_a;
+      *mb = g_maps[i].map_b;
+      return cudaSuccess;
+    }
+    const uint64_t age_i = g_maps[i].valid ? g_maps[i].stamp : 0;
+    const uint64_t age_v = g_maps[victim].valid ? g_maps[victim].stamp : 0;
+    if (age_i < age_v) victim = i;
+  }
+  MapEntry e{};
+  e.key = key;
+  cudaError_t err = make_tensor_map_3d(&e.map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, key.a,
+                                       (uint64_t)key.k, (uint64_t)key.m, (uint64_t)key.bsz, kTileK,
+                                       kTileM, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (err != cudaSuccess) return err;
+  err = make_tensor_map_3d(&e.map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, key.b, (uint64_t)key.n,
+                           (uint64_t)key.k, (uint64_t)key.bsz, 64, kTileK,
+                           CU_TENSOR_MAP_SWIZZLE_128B);
+  if (err != cudaSuccess) return err;
+  e.stamp = ++g_stamp;
+  e.valid = true;
+  g_maps[victim] = e;
+  *ma = e.map_a;
+  *mb = e.map_b;
+  return cudaSuccess;
+}
+
+}  // namespace
+
+bool gemm_shape_supported(int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
+                          const void* B, const void* C) {
+  if (b <= 0 || m <= 0 || k <= 0 || n <= 0) return false;
+  if (k % 8 || n % 8) return false;  // TMA row pitches must be multiples of 16 bytes
+  if (reinterpret_cast<uintptr_t>(A) % 16 || reinterpret_cast<uintptr_t>(B) % 16 ||
+      reinterpret_cast<uintptr_t>(C) % 16)
+    return false;
+  // Tensor-map extents are 32-bit, tile coordinates are ints.
+  if (m >= (1ll << 31) || n >= (1ll << 31) || k >= (1ll << 31) || b >= (1ll << 31)) return false;
+  return true;
+}
+
+GemmPlan gemm_plan(int, int64_t, int64_t, int64_t, int64_t, int) { return GemmPlan{true, 1, 0}; }
+
+cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan&, int64_t b, int64_t m, int64_t k,
+                        int64_t n, const uint16_t* A, const uint16_t* B, float* C, float*,
+                        cudaStream_t stream, uint64_t* launches) {
+  CUtensorMap map_a, map_b;
+  cudaError_t e = get_maps(MapKey{A, B, b, m, k, n}, &map_a, &map_b);
+  if (e != cudaSuccess) return e;
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [] {
+    attr_err = cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)kSmemBytes);
+  });
+  if (attr_err != cudaSuccess) return attr_err;
+
+  GemmParams p{};
+  p.C = C;
+  p.m = m; p.n = n; p.k = k;
+  p.c_batch = m * n;
+  p.m_tiles = (int)((m + kTileM - 1) / kTileM);
+  p.n_tiles = (int)((n + kTileN - 1) / kTileN);
+  p.tiles = b * p.m_tiles * (int64_t)p.n_tiles;
+  p.k_blocks = (int)((k + kTileK - 1) / kTileK);
+  p.status = dev.status;
+
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)std::min<int64_t>(p.tiles, dev.sms), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  e = cudaLaunchKernelEx(&cfg, gemm_kernel, map_a, map_b, p);
+  if (e == cudaSuccess) ++*launches;
+  return e;
 }
 
 }  // namespace morello

@@ -39,6 +39,7 @@ struct SkinnyParams {
   int col_blocks;
   int split_k;
   int k_chunk;
+  int early_b;  // 1: B may be fetched before the preceding kernel on the stream has completed
 };
 
 template <int M_T>
@@ -110,10 +111,16 @@ __device__ __forceinline__ void fma_row(float (&acc)[M_T][VEC], const float* __r
   }
 }
 
-template <int M_T, int VEC>
-__global__ void __launch_bounds__(Tuning<M_T>::kThreads)
+// Programmatic dependent launch: a kernel launched with the stream-serialisation
+// attribute may start while its predecessor drains; it must not touch global
+// memory before pdl_wait() returns (the predecessor has then completed and its
+// writes are visible).  pdl_release() lets the successor's blocks be scheduled.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;"); }
+
+template <int M_T, int VEC, int UNROLL, int THREADS>
+__global__ void __launch_bounds__(THREADS)
 skinny_kernel(const SkinnyParams p) {
-  constexpr int UNROLL = Tuning<M_T>::kUnroll;
   extern __shared__ __align__(16) float smem[];
   float* a_s = smem;                                  // [k_chunk][M_T]
   float* red = smem + (size_t)p.k_chunk * M_T;        // [row_lanes][M_T * units * VEC]
@@ -129,6 +136,7 @@ skinny_kernel(const SkinnyParams p) {
   const int64_t k0 = (int64_t)s * p.k_per_split;
   const int64_t k1 = min(p.k, k0 + p.k_per_split);
   const int R = p.row_lanes;
+  const int64_t step = (int64_t)R * p.n;
 
   float acc[M_T][VEC];
 #pragma unroll
@@ -137,7 +145,24 @@ skinny_kernel(const SkinnyParams p) {
     for (int j = 0; j < VEC; ++j) acc[i][j] = 0.f;
 
   const uint16_t* a_base = p.A + (int64_t)bb * p.a_batch;
-  const uint16_t* b_base = p.B + (int64_t)bb * p.b_batch + (int64_t)unit * VEC;
+  const uint16_t* bp = p.B + (int64_t)bb * p.b_batch + (int64_t)unit * VEC + (k0 + rl) * p.n;
+
+  // The first group of B rows is requested before A is staged, so that the
+  // staging latency hides under the first HBM round trip.  When the caller has
+  // declared B stable (early_b), it is requested even before the preceding
+  // kernel on the stream is known to have completed; A, C and the partial sums
+  // are only touched after pdl_wait().
+  BVec<VEC> v[UNROLL];
+  bool preloaded = false;
+  if (p.early_b) pdl_release(); else pdl_wait();
+  if (active) {
+    const int kcl0 = (int)min((int64_t)p.k_chunk, k1 - k0);
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u)
+      if (rl + u * R < kcl0) v[u].load(bp + u * step);
+    preloaded = true;
+  }
+  if (p.early_b) pdl_wait(); else pdl_release();
 
   for (int64_t kc0 = k0; kc0 < k1; kc0 += p.k_chunk) {
     const int kcl = (int)min((int64_t)p.k_chunk, k1 - kc0);
@@ -145,30 +170,29 @@ skinny_kernel(const SkinnyParams p) {
 #pragma unroll
     for (int i = 0; i < M_T; ++i) {
       for (int q = t; q < kcl; q += blockDim.x) {
-        const float v = (i < p.m)
+        const float av = (i < p.m)
             ? __uint_as_float(((uint32_t)a_base[(int64_t)i * p.k + kc0 + q]) << 16) : 0.f;
-        a_s[q * M_T + i] = v;
+        a_s[q * M_T + i] = av;
       }
     }
     __syncthreads();
     if (active) {
-      const uint16_t* bp = b_base + (kc0 + rl) * p.n;
-      const int64_t step = (int64_t)R * p.n;
-      int q = rl;
-      for (; q + (UNROLL - 1) * R < kcl; q += UNROLL * R) {
-        BVec<VEC> v[UNROLL];
+      // Rows q, q + R, ... of the chunk in groups of UNROLL: all loads of a group are
+      // issued before the first is consumed; rows past the chunk are predicated off.
+      for (int q = rl; q < kcl; q += UNROLL * R) {
+        if (!preloaded) {
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) v[u].load(bp + u * step);
+          for (int u = 0; u < UNROLL; ++u)
+            if (q + u * R < kcl) v[u].load(bp + u * step);
+        }
+        preloaded = false;
         bp += UNROLL * step;
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) fma_row<M_T, VEC>(acc, a_s + (q + u * R) * M_T, v[u]);
+        for (int u = 0; u < UNROLL; ++u)
+          if (q + u * R < kcl) fma_row<M_T, VEC>(acc, a_s + (q + u * R) * M_T, v[u]);
       }
-      for (; q < kcl; q += R) {
-        BVec<VEC> v;
-        v.load(bp);
-        bp += step;
-        fma_row<M_T, VEC>(acc, a_s + q * M_T, v);
-      }
+      // bp now points UNROLL*R-aligned past the chunk; rebase to the next chunk's first row.
+      bp = p.B + (int64_t)bb * p.b_batch + (int64_t)unit * VEC + (kc0 + kcl + rl) * p.n;
     }
   }
 
@@ -204,6 +228,8 @@ __global__ void __launch_bounds__(256)
 reduce_kernel(const float* __restrict__ partial, float* __restrict__ C, int64_t total,
               int64_t mn, int64_t c_batch, int split_k) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  pdl_wait();
+  pdl_release();
   if (idx >= total) return;
   float sum = partial[idx];
   for (int s = 1; s < split_k; ++s) sum += partial[(int64_t)s * total + idx];
@@ -212,18 +238,34 @@ reduce_kernel(const float* __restrict__ partial, float* __restrict__ C, int64_t 
   *c = *c + sum;
 }
 
+// Launch with programmatic stream serialisation (see pdl_wait above).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, int threads, size_t smem,
+                       cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3((unsigned)threads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 template <int M_T, int VEC>
 cudaError_t launch_one(const SkinnyPlan& plan, const SkinnyParams& prm, int64_t b,
                        cudaStream_t stream) {
-  auto kern = skinny_kernel<M_T, VEC>;
+  auto kern = skinny_kernel<M_T, VEC, Tuning<M_T>::kUnroll, Tuning<M_T>::kThreads>;
   if (plan.smem_bytes > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)plan.smem_bytes);
     if (e != cudaSuccess) return e;
   }
   dim3 grid((unsigned)(plan.col_blocks * plan.split_k), (unsigned)b, 1);
-  kern<<<grid, plan.threads, plan.smem_bytes, stream>>>(prm);
-  return cudaGetLastError();
+  return launch_pdl(kern, grid, plan.threads, plan.smem_bytes, stream, prm);
 }
 
 template <int M_T>
@@ -338,9 +380,9 @@ cudaError_t skinny_launch(const SkinnyPlan& plan, int64_t b, int m, int64_t k, i
   if (plan.split_k > 1) {
     const int64_t total = b * m * n;
     const int64_t blocks = (total + 255) / 256;
-    reduce_kernel<<<(unsigned)blocks, 256, 0, stream>>>(workspace, C, total, (int64_t)m * n,
-                                                        c_batch, plan.split_k);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_pdl(reduce_kernel, dim3((unsigned)blocks, 1, 1), 256, 0, stream,
+                               (const float*)workspace, C, total, (int64_t)m * n, c_batch,
+                               plan.split_k);
     if (e != cudaSuccess) return e;
     ++*launches;
   }

@@ -67,6 +67,9 @@ def test_selector_is_shape_based(mb):
     assert mb.morello_select_path(1, 4, 4, 16) == mb.MORELLO_PATH_SKINNY
     assert mb.morello_select_path(1, 16, 2048, 16384) == mb.MORELLO_PATH_SKINNY
     assert mb.morello_select_path(1, 4096, 4096, 4095) == mb.MORELLO_PATH_SKINNY   # n % 8 != 0
+    assert mb.morello_select_path(1, 4096, 4096, 4096) == mb.MORELLO_PATH_TCGEN05
+    assert mb.morello_select_path(8, 2048, 2048, 16384) == mb.MORELLO_PATH_TCGEN05
+    assert mb.morello_select_path(1, 17, 8, 8) == mb.MORELLO_PATH_TCGEN05
     assert mb.morello_select_path(1, -1, 4, 4) == -1
 
 

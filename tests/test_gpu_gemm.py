@@ -1,0 +1,100 @@
+"""GPU parity of the tcgen05 tensor-core path (forced through the C ABI) against
+the CPU oracle: single tiles first, then ragged edges, batches, operand-layout pins
+and the cross-check against the FP32-FMA path."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2505_01637_b200 import binding as mb
+from paper_2505_01637_b200 import workloads as w
+
+from gpu_util import assert_bit_exact, bits, check_full, gpu_run
+
+pytestmark = pytest.mark.gpu
+TC = mb.MORELLO_PATH_TCGEN05
+
+
+@pytest.mark.parametrize("shape", [
+    (1, 128, 64, 256),      # exactly one tile, one k block
+    (1, 128, 16, 256),      # one MMA instruction's worth of k
+    (1, 128, 256, 256),     # one tile, the stage ring wraps once
+    (1, 128, 640, 256),     # ring wraps several times
+    (1, 256, 128, 512),     # 2 x 2 tiles
+    (1, 17, 8, 8),          # smallest shape the selector sends here
+    (1, 100, 72, 200),      # ragged m, k, n inside one tile
+    (1, 129, 200, 264),     # one row / one 8-column group into the next tile
+    (2, 300, 520, 776),     # batches with ragged everything
+    (3, 64, 64, 64),
+    (1, 1024, 128, 2048),   # more tiles than fit one wave of a small grid
+])
+def test_integer_inputs_bit_exact(shape):
+    b, m, k, n = shape
+    A, B, C = w.make(b, m, k, n, seed=sum(shape), ab="int4", c="normal")
+    check_full(A, B, C, integer=True, path=TC, what="tcgen05 %s" % (shape,))
+
+
+def test_one_hot_operands_pin_the_operand_layouts():
+    b, m, k, n = 2, 160, 136, 328
+    rng = np.random.default_rng(0)
+    Bv = rng.integers(-100, 101, size=(b, k, n)).astype(np.float32)
+    Av = rng.integers(-100, 101, size=(b, m, k)).astype(np.float32)
+    C = rng.integers(-50, 51, size=(b, m, n)).astype(np.float32)
+    for (b0, i0, p0) in [(0, 0, 0), (0, 37, 70), (1, 159, 135), (1, 128, 64)]:
+        A1 = np.zeros((b, m, k), np.float32)
+        A1[b0, i0, p0] = 2.0
+        want = C.copy()
+        want[b0, i0, :] += 2.0 * Bv[b0, p0, :]
+        got = gpu_run(w.f32_to_bf16_rne(A1), w.f32_to_bf16_rne(Bv), C, path=TC)
+        assert_bit_exact(got, want, "one-hot A at %s" % ((b0, i0, p0),))
+    for (b0, p0, j0) in [(0, 0, 0), (0, 70, 201), (1, 135, 327), (1, 64, 256)]:
+        B1 = np.zeros((b, k, n), np.float32)
+        B1[b0, p0, j0] = -3.0
+        want = C.copy()
+        want[b0, :, j0] += -3.0 * Av[b0, :, p0]
+        got = gpu_run(w.f32_to_bf16_rne(Av), w.f32_to_bf16_rne(B1), C, path=TC)
+        assert_bit_exact(got, want, "one-hot B at %s" % ((b0, p0, j0),))
+
+
+def test_identity_operands():
+    d = 192
+    rng = np.random.default_rng(1)
+    X = rng.integers(-100, 101, size=(1, d, d)).astype(np.float32)
+    I = np.eye(d, dtype=np.float32)[None]
+    C = rng.standard_normal((1, d, d)).astype(np.float32)
+    want = (C.astype(np.float64) + X).astype(np.float32)
+    assert_bit_exact(gpu_run(w.f32_to_bf16_rne(I), w.f32_to_bf16_rne(X), C, path=TC), want, "A = I")
+    assert_bit_exact(gpu_run(w.f32_to_bf16_rne(X), w.f32_to_bf16_rne(I), C, path=TC), want, "B = I")
+
+
+@pytest.mark.parametrize("shape", [(1, 256, 512, 512), (2, 200, 1000, 328), (1, 128, 4096, 256),
+                                   (1, 2048, 2048, 512)])
+def test_random_inputs_within_tolerance(shape):
+    b, m, k, n = shape
+    for ab, c in (("uniform", "normal"), ("normal_rsqrtk", "normal0.1")):
+        A, B, C = w.make(b, m, k, n, seed=sum(shape), ab=ab, c=c)
+        check_full(A, B, C, integer=False, path=TC, what="tcgen05 %s %s" % (shape, ab))
+
+
+@pytest.mark.parametrize("shape", [(1, 16, 512, 1024), (2, 8, 264, 520), (1, 48, 128, 256)])
+def test_both_kernel_families_agree(shape):
+    b, m, k, n = shape
+    A, B, C = w.make(b, m, k, n, seed=3, ab="int4", c="normal")
+    fma = gpu_run(A, B, C, path=mb.MORELLO_PATH_SKINNY)
+    tc = gpu_run(A, B, C, path=TC)
+    assert_bit_exact(tc, fma, "tcgen05 vs skinny on integers %s" % (shape,))
+    A, B, C = w.make(b, m, k, n, seed=4, ab="uniform", c="normal")
+    fma = gpu_run(A, B, C, path=mb.MORELLO_PATH_SKINNY)
+    tc = gpu_run(A, B, C, path=TC)
+    T = oracle.abs_dot(b, m, k, n, A, B)
+    assert np.all(np.abs(fma.astype(np.float64) - tc) <= 2 * (1e-5 * T + 1e-6))
+
+
+def test_repeated_calls_give_identical_bits_and_accumulate():
+    b, m, k, n = 1, 384, 1024, 768
+    A, B, C = w.make(b, m, k, n, seed=5, ab="normal_rsqrtk", c="normal")
+    first = gpu_run(A, B, C, path=TC)
+    for _ in range(3):
+        assert np.array_equal(bits(gpu_run(A, B, C, path=TC)), bits(first))
+    A, B, C = w.make(b, m, k, n, seed=6, ab="int4", c="int8")
+    twice = oracle.matmul_accum(b, m, k, n, A, B, oracle.matmul_accum(b, m, k, n, A, B, C))
+    assert_bit_exact(gpu_run(A, B, C, path=TC, calls=2), twice, "two accumulating calls")
