@@ -99,6 +99,39 @@ int morello_matmul_accum_ws(int64_t b, int64_t m, int64_t k, int64_t n,
 int morello_matmul_accum_host(int64_t b, int64_t m, int64_t k, int64_t n,
                               const void* A_host, const void* B_host, float* C_host);
 
+/*
+ * Allocation-free variant (the paper has no counterpart: this exists for callers,
+ * not for the method).  Same operation, computed by the FP32-FMA kernel with the k
+ * range cut into `split_k` slices (0 = let the library choose); the slices' partial
+ * sums go to a fixed device array of MORELLO_NOALLOC_SCRATCH_BYTES that is part of
+ * the library image, so neither this call nor anything it uses ever calls cudaMalloc,
+ * cudaFree or an allocating library routine.  It is meant for processes that must not
+ * allocate at call time: ones that gave all device memory to their own pool at
+ * start-up (a late cudaMalloc may fail there, and while it runs it holds up every
+ * stream of the process), or ones barred from growing their footprint once serving.
+ *
+ * Limits and rules:
+ *  - the partial sums, split_k * b * min(m, 16) * n * 4 bytes, must fit the array;
+ *    otherwise MORELLO_ERR_WORKSPACE is returned and nothing is enqueued
+ *    (split_k = 1 needs no scratch and always fits);
+ *  - the first call on each device resolves the array's device address (with that
+ *    device current) and queries two device attributes; make that first call before
+ *    starting any stream capture;
+ *  - all calls on a device share the one array and it keeps whatever the last call
+ *    left in it.  Nothing in it has to be zero beforehand (every word that is read was
+ *    written by the same call), but two calls that overlap on the GPU -- different
+ *    streams, or one stream of each of two host threads -- race on it: serialise them;
+ *  - every GPU that loads the library holds the array until the process exits.
+ * Otherwise as morello_matmul_accum: device pointers, asynchronous on `stream`, same
+ * status codes, deterministic for a given shape and split.
+ */
+#define MORELLO_NOALLOC_SCRATCH_BYTES (4u << 20)
+int morello_matmul_accum_noalloc(int split_k, int64_t b, int64_t m, int64_t k, int64_t n,
+                                 const void* A, const void* B, float* C, void* stream);
+
+/* MORELLO_NOALLOC_SCRATCH_BYTES as the loaded library was built with. */
+size_t morello_noalloc_scratch_limit(void);
+
 /* --- introspection and experiments (tests and benchmarks) ------------------ */
 
 /* The path the selector picks for this shape with 16-byte-aligned operands:

@@ -37,6 +37,8 @@ SIGNATURES = {
     "morello_workspace_bytes": (_sz, [_i64, _i64, _i64, _i64]),
     "morello_matmul_accum_ws": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _sz, _vp]),
     "morello_matmul_accum_host": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp]),
+    "morello_matmul_accum_noalloc": (_int, [_int, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
+    "morello_noalloc_scratch_limit": (_sz, []),
     "morello_select_path": (_int, [_i64, _i64, _i64, _i64]),
     "morello_matmul_accum_forced": (_int, [_int, _int, _i64, _i64, _i64, _i64, _vp, _vp, _vp,
                                            _vp, _sz, _vp]),
@@ -124,6 +126,17 @@ def morello_matmul_accum_ws(b, m, k, n, A, B, C, workspace, workspace_bytes, str
 def morello_matmul_accum_host(b, m, k, n, A_host, B_host, C_host) -> None:
     _check(lib().morello_matmul_accum_host(b, m, k, n, _addr(A_host), _addr(B_host), _addr(C_host)),
            "morello_matmul_accum_host")
+
+
+def morello_matmul_accum_noalloc(split_k, b, m, k, n, A, B, C, stream=None) -> None:
+    """Allocation-free variant: partial sums live in a fixed array inside the library."""
+    _check(lib().morello_matmul_accum_noalloc(split_k, b, m, k, n, _addr(A), _addr(B), _addr(C),
+                                              _stream(stream)),
+           "morello_matmul_accum_noalloc")
+
+
+def morello_noalloc_scratch_limit() -> int:
+    return int(lib().morello_noalloc_scratch_limit())
 
 
 def morello_select_path(b, m, k, n) -> int:
