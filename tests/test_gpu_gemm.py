@@ -27,13 +27,15 @@ TC = mb.MORELLO_PATH_TCGEN05
     (3, 64, 64, 64),
     (1, 1024, 128, 2048),   # more tiles than fit one wave of a small grid
 ])
-def test_integer_inputs_bit_exact(shape):
+@pytest.mark.parametrize("form", [1, 2])      # one CTA per tile / a CTA pair per tile
+def test_integer_inputs_bit_exact(shape, form):
     b, m, k, n = shape
     A, B, C = w.make(b, m, k, n, seed=sum(shape), ab="int4", c="normal")
-    check_full(A, B, C, integer=True, path=TC, what="tcgen05 %s" % (shape,))
+    check_full(A, B, C, integer=True, path=TC, split_k=form, what="tcgen05 form %d %s" % (form, shape))
 
 
-def test_one_hot_operands_pin_the_operand_layouts():
+@pytest.mark.parametrize("form", [1, 2])
+def test_one_hot_operands_pin_the_operand_layouts(form):
     b, m, k, n = 2, 160, 136, 328
     rng = np.random.default_rng(0)
     Bv = rng.integers(-100, 101, size=(b, k, n)).astype(np.float32)
@@ -44,14 +46,14 @@ def test_one_hot_operands_pin_the_operand_layouts():
         A1[b0, i0, p0] = 2.0
         want = C.copy()
         want[b0, i0, :] += 2.0 * Bv[b0, p0, :]
-        got = gpu_run(w.f32_to_bf16_rne(A1), w.f32_to_bf16_rne(Bv), C, path=TC)
+        got = gpu_run(w.f32_to_bf16_rne(A1), w.f32_to_bf16_rne(Bv), C, path=TC, split_k=form)
         assert_bit_exact(got, want, "one-hot A at %s" % ((b0, i0, p0),))
     for (b0, p0, j0) in [(0, 0, 0), (0, 70, 201), (1, 135, 327), (1, 64, 256)]:
         B1 = np.zeros((b, k, n), np.float32)
         B1[b0, p0, j0] = -3.0
         want = C.copy()
         want[b0, :, j0] += -3.0 * Av[b0, :, p0]
-        got = gpu_run(w.f32_to_bf16_rne(Av), w.f32_to_bf16_rne(B1), C, path=TC)
+        got = gpu_run(w.f32_to_bf16_rne(Av), w.f32_to_bf16_rne(B1), C, path=TC, split_k=form)
         assert_bit_exact(got, want, "one-hot B at %s" % ((b0, p0, j0),))
 
 
@@ -68,11 +70,13 @@ def test_identity_operands():
 
 @pytest.mark.parametrize("shape", [(1, 256, 512, 512), (2, 200, 1000, 328), (1, 128, 4096, 256),
                                    (1, 2048, 2048, 512)])
-def test_random_inputs_within_tolerance(shape):
+@pytest.mark.parametrize("form", [1, 2])
+def test_random_inputs_within_tolerance(shape, form):
     b, m, k, n = shape
     for ab, c in (("uniform", "normal"), ("normal_rsqrtk", "normal0.1")):
         A, B, C = w.make(b, m, k, n, seed=sum(shape), ab=ab, c=c)
-        check_full(A, B, C, integer=False, path=TC, what="tcgen05 %s %s" % (shape, ab))
+        check_full(A, B, C, integer=False, path=TC, split_k=form,
+                   what="tcgen05 form %d %s %s" % (form, shape, ab))
 
 
 @pytest.mark.parametrize("shape", [(1, 16, 512, 1024), (2, 8, 264, 520), (1, 48, 128, 256)])
@@ -89,12 +93,13 @@ def test_both_kernel_families_agree(shape):
     assert np.all(np.abs(fma.astype(np.float64) - tc) <= 2 * (1e-5 * T + 1e-6))
 
 
-def test_repeated_calls_give_identical_bits_and_accumulate():
+@pytest.mark.parametrize("form", [1, 2])
+def test_repeated_calls_give_identical_bits_and_accumulate(form):
     b, m, k, n = 1, 384, 1024, 768
     A, B, C = w.make(b, m, k, n, seed=5, ab="normal_rsqrtk", c="normal")
-    first = gpu_run(A, B, C, path=TC)
+    first = gpu_run(A, B, C, path=TC, split_k=form)
     for _ in range(3):
-        assert np.array_equal(bits(gpu_run(A, B, C, path=TC)), bits(first))
+        assert np.array_equal(bits(gpu_run(A, B, C, path=TC, split_k=form)), bits(first))
     A, B, C = w.make(b, m, k, n, seed=6, ab="int4", c="int8")
     twice = oracle.matmul_accum(b, m, k, n, A, B, oracle.matmul_accum(b, m, k, n, A, B, C))
-    assert_bit_exact(gpu_run(A, B, C, path=TC, calls=2), twice, "two accumulating calls")
+    assert_bit_exact(gpu_run(A, B, C, path=TC, split_k=form, calls=2), twice, "two accumulating calls")
