@@ -220,7 +220,7 @@ def time_calls(torch, fn, steps, warmup):
     return start.elapsed_time(stop) * 1e-3
 
 
-def bench_config(torch, mb, idx, iters, warmup, peaks, windows, path=None):
+def bench_config(torch, mb, idx, iters, warmup, peaks, windows, path=None, split_k=0):
     """Device-timed throughput of one config (inputs resident, rotating when small)."""
     cfg = w.CONFIGS[idx]
     b, m, k, n = cfg.shape
@@ -242,7 +242,7 @@ def bench_config(torch, mb, idx, iters, warmup, peaks, windows, path=None):
 
     def step(i):
         pa, pb, pc = ptrs[i % sets]
-        rc = call(forced, 0, b, m, k, n, pa, pb, pc, None, 0, stream)
+        rc = call(forced, split_k, b, m, k, n, pa, pb, pc, None, 0, stream)
         if rc != 0:
             raise mb.MorelloError(rc, "bench %s" % cfg.name)
 
@@ -269,6 +269,25 @@ def bench_config(torch, mb, idx, iters, warmup, peaks, windows, path=None):
     del dev
     torch.cuda.empty_cache()
     return rec
+
+
+def run_case(args):
+    """One configuration alone, device-timed: the command the ncu captures under
+    profiles/ were taken with, and the unit of the sweeps quoted in the design notes."""
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(0)
+    from paper_2505_01637_b200 import binding as mb
+    mb.lib()
+    peaks, _ = load_peaks()
+    path = {"auto": None, "skinny": mb.MORELLO_PATH_SKINNY, "tcgen05": mb.MORELLO_PATH_TCGEN05}[args.path]
+    rec = bench_config(torch, mb, args.case - 1, args.steps, args.warmup, peaks, [], path=path,
+                       split_k=args.split)
+    rec["case"] = args.case
+    rec["split_k_knob"] = args.split
+    print(json.dumps(rec))
+    return 0
 
 
 def run_ours(args):
@@ -463,12 +482,19 @@ def main():
     ap.add_argument("--configs", default="1,3,4,5",
                     help="1-based extra configs to time at --gpus 1 ('' for none)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--case", type=int, default=0,
+                    help="time only this 1-based config (with --steps/--warmup calls) and print its record")
+    ap.add_argument("--path", default="auto", choices=["auto", "skinny", "tcgen05"],
+                    help="kernel family for --case")
+    ap.add_argument("--split", type=int, default=0, help="forced split / form knob for --case")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     args.steps = max(args.steps, 1)
     args.configs = [int(x) - 1 for x in args.configs.split(",") if x.strip()]
     if args.impl == "reference":
         return run_reference(args)
+    if args.case:
+        return run_case(args)
     return run_ours(args)
 
 

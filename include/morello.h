@@ -141,12 +141,14 @@ int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n);
 /*
  * Run on a given path (MORELLO_PATH_AUTO = selector) with a given split of the
  * k range across thread blocks (0 = automatic).  On the tcgen05 path, which never
- * splits k, the argument instead selects the tile form: 0 = by shape, 1 = one CTA per
- * 128 x 256 tile, 2 = a pair of CTAs per 256 x 256 tile (cta_group::2).  Returns
- * MORELLO_ERR_UNSUPPORTED_PATH, and enqueues nothing, when the path cannot run
- * the shape (the tcgen05 path needs k % 8 == 0, n % 8 == 0 and 16-byte-aligned
- * A, B, C).  workspace may be NULL with workspace_bytes 0 to use the library's
- * own per-device scratch.
+ * splits k, the argument instead selects the tile: (value % 16) is the form -- 0 = by
+ * shape, 1 = one CTA per 128-row tile, 2 = a pair of CTAs per 256-row tile
+ * (cta_group::2) -- and (value / 16) is the tile's column count / 64 -- 0 = by shape,
+ * 1, 2 or 4 (64 columns only with form 1).  Returns MORELLO_ERR_UNSUPPORTED_PATH, and
+ * enqueues nothing, when the path cannot run the shape (the tcgen05 path needs
+ * k % 8 == 0, n % 8 == 0 and 16-byte-aligned A, B, C) or the value names no tile.
+ * workspace may be NULL with workspace_bytes 0 to use the library's own per-device
+ * scratch.
  */
 int morello_matmul_accum_forced(int path, int split_k,
                                 int64_t b, int64_t m, int64_t k, int64_t n,

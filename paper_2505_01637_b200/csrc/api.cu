@@ -169,6 +169,7 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
   cudaError_t e = cudaSuccess;
   if (path == MORELLO_PATH_TCGEN05) {
     const GemmPlan plan = gemm_plan(sms, b, m, k, n, split_k);
+    if (!plan.supported) return MORELLO_ERR_UNSUPPORTED_PATH;
     e = gemm_launch(st->info, plan, b, m, k, n, static_cast<const uint16_t*>(A),
                     static_cast<const uint16_t*>(B), C, ws, s, &launches);
   } else {

@@ -1,21 +1,27 @@
 // Tensor-core MatmulAccum for sm_100a: C[b] += A[b] x B[b] with bf16 operands and
 // f32 accumulation in tensor memory.
 //
-// One persistent thread block per SM walks 128 x 256 output tiles.  Its warps are
-// specialised:
-//   warp 0   producer: TMA loads of a 128 x 64 tile of A and a 64 x 256 tile of B per
-//            k block into a ring of shared-memory stages (128-byte swizzle);
-//   warp 1   MMA issuer: one elected lane issues tcgen05.mma (M 128, N 256, K 16), four
-//            per k block, accumulating in one of two 256-column TMEM buffers, and
-//            commits to the stage's "empty" barrier and, after the last k block, to the
-//            buffer's "full" barrier;
+// Persistent thread blocks (one per SM) walk output tiles.  Two forms:
+//   one CTA per tile   (cta_group::1): tile 128 x N, N in {64, 128, 256};
+//   a CTA pair per tile (cta_group::2): tile 256 x N, N in {128, 256}; CTA r of the
+//       pair holds rows [128 r, 128 r + 128) of A and columns [N/2 r, N/2 r + N/2) of B,
+//       the leader (r = 0) issues the MMAs for both, each CTA drains its own 128 rows.
+// Warps are specialised:
+//   warp 0   producer: TMA loads of a 128 x 64 tile of A and a 64 x (N or N/2) tile of B
+//            per k block into a ring of shared-memory stages (128-byte swizzle);
+//   warp 1   MMA issuer: one elected lane issues tcgen05.mma (K 16), four per k block,
+//            accumulating in one of two TMEM buffers, and commits to the stage's "empty"
+//            barrier and, after the last k block, to the buffer's "full" barrier;
 //   warps 2-5 epilogue: read the accumulator with tcgen05.ld (each warp its own 32-lane
-//            quarter), add it to C in global memory (one rounding per element), and hand
-//            the buffer back.  The epilogue of tile i overlaps the main loop of tile i+1.
+//            quarter) 32 columns at a time, park the 32 x 32 block in shared memory in
+//            the 128-byte-swizzled layout and hand it to the TMA engine as a reduce-add
+//            into C (cp.reduce.async.bulk.tensor ... add.f32): one addition per element,
+//            performed in L2, nothing read back by the SM.  The epilogue of tile i
+//            overlaps the main loop of tile i+1.
 // A is [m][k] (K-major operand).  B is [k][n], i.e. N is contiguous: it is fed as an
 // MN-major operand, each 64-column group of the tile being one TMA box of 64 k rows.
-// Rows, columns and k blocks past the tensor edge are zero-filled by TMA and the
-// epilogue predicates its accesses, so m, n and k need not be multiples of the tile.
+// Rows, columns and k blocks past the tensor edge are zero-filled by the TMA loads and
+// clipped by the TMA reduce, so m, n and k need not be multiples of the tile.
 // Every barrier wait is bounded (sm100::mbar_wait); on a timeout the block stops
 // issuing work, records a status word and exits after releasing its TMEM.
 #include <algorithm>
@@ -31,31 +37,31 @@ namespace {
 using namespace sm100;
 
 constexpr int kRowsPerCta = 128;                   // accumulator rows (TMEM lanes) per CTA
-constexpr int kTileN = 256;                        // accumulator columns per tile
 constexpr int kTileK = 64;                         // one 128-byte swizzle span of bf16
 constexpr int kBytesA = kRowsPerCta * kTileK * 2;  // 16 KiB
 constexpr int kBoxBytesB = kTileK * 64 * 2;        // one TMA box of B: 64 k rows x 64 columns
-constexpr int kAccColumns = kTileN;                // f32 columns per accumulator buffer
-constexpr int kTmemColumns = 2 * kAccColumns;      // 512: the whole tensor memory
+constexpr int kAccStride = 256;                    // TMEM columns between the two accumulators
+constexpr int kTmemColumns = 2 * kAccStride;       // 512: the whole tensor memory
 constexpr int kThreads = 192;
-constexpr int kMaxStages = 6;
+constexpr int kMaxStages = 8;
+constexpr int kEpiCols = 32;                       // columns per epilogue block (128 bytes of f32)
+constexpr int kEpiBlockBytes = 32 * kEpiCols * 4;  // one warp's 32 x 32 block
+constexpr int kEpiBytes = 4 * 2 * kEpiBlockBytes;  // 4 warps x 2 blocks in flight
+constexpr int kSmemBudget = 227 * 1024;
 
-// kPair = false: one CTA per 128 x 256 tile (cta_group::1), B tile whole in its
-// shared memory.  kPair = true: two CTAs of a cluster share a 256 x 256 tile
-// (cta_group::2): CTA r holds rows [128 r, 128 r + 128) of A and columns
-// [128 r, 128 r + 128) of B, the leader (r = 0) issues the MMAs for both, and each
-// CTA's epilogue drains its own 128 rows.  Halving B per CTA halves both the TMA fill
-// and the operand reads of shared memory per MMA, which is what bounds the 1-CTA form.
-template <bool kPair>
+template <bool kPair, int kTileN>
 struct Shape {
   static constexpr int kCtas = kPair ? 2 : 1;
   static constexpr int kTileM = kRowsPerCta * kCtas;
   static constexpr int kColsB = kTileN / kCtas;          // columns of B held per CTA
   static constexpr int kBoxesB = kColsB / 64;
   static constexpr int kBytesB = kTileK * kColsB * 2;
-  static constexpr int kStageBytes = kBytesA + kBytesB;  // 48 KiB / 32 KiB
-  static constexpr int kStages = kPair ? 6 : 4;
-  static constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256;
+  static constexpr int kStageBytes = kBytesA + kBytesB;
+  static constexpr int kFit = (kSmemBudget - kEpiBytes - 1024 - 256) / kStageBytes;
+  static constexpr int kStages = kFit < kMaxStages ? kFit : kMaxStages;
+  static constexpr size_t kSmemBytes =
+      (size_t)kStages * kStageBytes + kEpiBytes + 1024 /*alignment slack*/ + 256;
+  static_assert(kColsB % 64 == 0 && kTileN <= kAccStride, "tile shape");
 };
 
 struct GemmParams {
@@ -77,18 +83,19 @@ struct Barriers {
   int abort_flag;
 };
 
-template <bool kPair>
+template <bool kPair, int kTileN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-            const GemmParams p) {
-  using S = Shape<kPair>;
+            const __grid_constant__ CUtensorMap map_c, const GemmParams p) {
+  using S = Shape<kPair, kTileN>;
   extern __shared__ uint8_t smem_raw[];
   // Stage buffers must sit on 1024-byte boundaries (the swizzle pattern repeats every
   // 8 rows of 128 bytes and is keyed on address bits 7-9).  The carve-up is identical in
   // both CTAs of a pair: the pair MMA addresses the peer's operands by the same offsets.
   uint8_t* stages = reinterpret_cast<uint8_t*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  Barriers* bars = reinterpret_cast<Barriers*>(stages + (size_t)S::kStages * S::kStageBytes);
+  uint8_t* epi = stages + (size_t)S::kStages * S::kStageBytes;   // 1024-byte aligned as well
+  Barriers* bars = reinterpret_cast<Barriers*>(epi + kEpiBytes);
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5;
@@ -110,6 +117,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     mbar_fence_init();
     tma_prefetch_descriptor(&map_a);
     tma_prefetch_descriptor(&map_b);
+    tma_prefetch_descriptor(&map_c);
   }
   if (warp == 1) {
     if constexpr (kPair) {
@@ -178,7 +186,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       for (int64_t t = unit; t < p.tiles && ok; t += units) {
         if (!(ok = mbar_wait(&bars->acc_empty[buf], acc_phase ^ 1, abort_flag, p.status, 2))) break;
         tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + (uint32_t)buf * kAccColumns;
+        const uint32_t d_tmem = tmem_base + (uint32_t)buf * kAccStride;
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!(ok = mbar_wait(&bars->full[stage], phase, abort_flag, p.status, 3))) break;
           tc_fence_after_sync();
@@ -208,29 +216,41 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   } else {
     // ------------------------------------------------------------------ epilogue
     const int quarter = warp & 3;  // TMEM lanes [32 * quarter, 32 * quarter + 32)
+    uint8_t* my_blocks = epi + (size_t)quarter * 2 * kEpiBlockBytes;
+    // Row `lane` of a block is 128 bytes; its 16-byte chunk j sits at chunk j ^ (lane % 8)
+    // (the 128-byte swizzle the tensor map of C expects), which also spreads a quarter
+    // warp's stores over all banks.
+    const uint32_t row_off = (uint32_t)lane * 128u;
+    const uint32_t sw = (uint32_t)(lane & 7);
     int buf = 0;
     uint32_t acc_phase = 0;
+    uint32_t blk = 0;              // alternates between this warp's two blocks
     bool ok = true;
     for (int64_t t = unit; t < p.tiles && ok; t += units) {
       const int mt = (int)(t % p.m_tiles);
       const int nt = (int)((t / p.m_tiles) % p.n_tiles);
-      const int64_t bb = t / ((int64_t)p.m_tiles * p.n_tiles);
+      const int bb = (int)(t / ((int64_t)p.m_tiles * p.n_tiles));
       ok = mbar_wait(&bars->acc_full[buf], acc_phase, abort_flag, p.status, 4);
       ok = __all_sync(0xffffffffu, ok);  // also reconverges the warp for the aligned TMEM loads
       if (!ok) break;
       tc_fence_after_sync();
-      const int64_t row = (int64_t)mt * S::kTileM + (int64_t)rank * kRowsPerCta + quarter * 32 + lane;
-      const int64_t col0 = (int64_t)nt * kTileN;
-      float* crow = p.C + bb * p.c_batch + row * p.n + col0;
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * kAccColumns;
+      const int row0 = mt * S::kTileM + (int)rank * kRowsPerCta + quarter * 32;
+      const int col0 = nt * kTileN;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * kAccStride;
+      const bool rows_live = row0 < p.m;   // warp-uniform
 #pragma unroll 1
-      for (int c = 0; c < kTileN; c += 64) {
-        uint32_t r0[32], r1[32];
-        tmem_ld_32x32(taddr + c, r0);
-        tmem_ld_32x32(taddr + c + 32, r1);
-        tmem_ld_wait();
-        if (c + 64 == kTileN) {
-          // The accumulator is in registers: hand the buffer back before the global traffic.
+      for (int c = 0; c < kTileN; c += kEpiCols) {
+        const bool live = rows_live && (col0 + c < p.n);
+        uint32_t r[32];
+        if (live) {
+          // The block written two steps ago must have been read by the TMA engine.
+          if (lane == 0) bulk_wait_group_read<1>();
+          __syncwarp();
+          tmem_ld_32x32(taddr + c, r);
+          tmem_ld_wait();
+        }
+        if (c + kEpiCols == kTileN) {
+          // The accumulator has left tensor memory: hand the buffer back to the MMA issuer.
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) {
@@ -238,22 +258,28 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             else mbar_arrive(&bars->acc_empty[buf]);
           }
         }
-        if (row < p.m) {
-          // C += acc: one reduction per element per call, performed at L2 (n % 4 == 0 here).
+        if (live) {
+          const uint32_t dst = smem_u32(my_blocks + blk * kEpiBlockBytes) + row_off;
 #pragma unroll
-          for (int j = 0; j < 32; j += 4)
-            if (col0 + c + j < p.n)
-              red_add_v4(crow + c + j, __uint_as_float(r0[j]), __uint_as_float(r0[j + 1]),
-                         __uint_as_float(r0[j + 2]), __uint_as_float(r0[j + 3]));
-#pragma unroll
-          for (int j = 0; j < 32; j += 4)
-            if (col0 + c + 32 + j < p.n)
-              red_add_v4(crow + c + 32 + j, __uint_as_float(r1[j]), __uint_as_float(r1[j + 1]),
-                         __uint_as_float(r1[j + 2]), __uint_as_float(r1[j + 3]));
+          for (int j = 0; j < 8; ++j)
+            st_shared_v4(dst + (((uint32_t)j ^ sw) << 4), r[4 * j], r[4 * j + 1], r[4 * j + 2],
+                         r[4 * j + 3]);
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            // C[bb, row0 : row0 + 32, col0 + c : col0 + c + 32] += block; rows and columns
+            // past the edge of C are dropped by the TMA engine.
+            tma_reduce_add_3d(&map_c, my_blocks + blk * kEpiBlockBytes, col0 + c, row0, bb);
+            bulk_commit_group();
+          }
+          blk ^= 1u;
         }
       }
       if (++buf == 2) { buf = 0; acc_phase ^= 1; }
     }
+    // Shared memory must outlive the engine's reads, and the additions must have been
+    // performed before the kernel counts as complete.
+    if (lane == 0) bulk_wait_group<0>();
   }
 
   __syncwarp();  // the elected lanes rejoin their warps before the aligned barriers below
@@ -271,27 +297,28 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   }
 }
 
-// Tensor maps are cached per (pointer, shape): encoding one costs a few microseconds.
+// Tensor maps are cached per (pointers, shape): encoding one costs a few microseconds.
 struct MapKey {
   const void* a;
   const void* b;
+  const void* c;
   int64_t bsz, m, k, n;
   bool operator==(const MapKey& o) const {
-    return a == o.a && b == o.b && bsz == o.bsz && m == o.m && k == o.k && n == o.n;
+    return a == o.a && b == o.b && c == o.c && bsz == o.bsz && m == o.m && k == o.k && n == o.n;
   }
 };
 struct MapEntry {
   MapKey key;
-  CUtensorMap map_a, map_b;
+  CUtensorMap map_a, map_b, map_c;
   uint64_t stamp;
   bool valid;
 };
-constexpr int kMapCache = 32;
+constexpr int kMapCache = 64;
 MapEntry g_maps[kMapCache];
 uint64_t g_stamp = 0;
 std::mutex g_map_mutex;
 
-cudaError_t get_maps(const MapKey& key, CUtensorMap* ma, CUtensorMap* mb) {
+cudaError_t get_maps(const MapKey& key, CUtensorMap* ma, CUtensorMap* mb, CUtensorMap* mc) {
   std::lock_guard<std::mutex> lock(g_map_mutex);
   int victim = 0;   // an unused slot if there is one, else the least recently used
   for (int i = 0; i < kMapCache; ++i) {
@@ -299,6 +326,7 @@ cudaError_t get_maps(const MapKey& key, CUtensorMap* ma, CUtensorMap* mb) {
       g_maps[i].stamp = ++g_stamp;
       *ma = g_maps[i].map_a;
       *mb = g_maps[i].map_b;
+      *mc = g_maps[i].map_c;
       return cudaSuccess;
     }
     const uint64_t age_i = g_maps[i].valid ? g_maps[i].stamp : 0;
@@ -315,11 +343,16 @@ cudaError_t get_maps(const MapKey& key, CUtensorMap* ma, CUtensorMap* mb) {
                            (uint64_t)key.k, (uint64_t)key.bsz, 64, kTileK,
                            CU_TENSOR_MAP_SWIZZLE_128B);
   if (err != cudaSuccess) return err;
+  err = make_tensor_map_3d(&e.map_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, key.c, (uint64_t)key.n,
+                           (uint64_t)key.m, (uint64_t)key.bsz, kEpiCols, 32,
+                           CU_TENSOR_MAP_SWIZZLE_128B);
+  if (err != cudaSuccess) return err;
   e.stamp = ++g_stamp;
   e.valid = true;
   g_maps[victim] = e;
   *ma = e.map_a;
   *mb = e.map_b;
+  *mc = e.map_c;
   return cudaSuccess;
 }
 
@@ -337,25 +370,49 @@ bool gemm_shape_supported(int64_t b, int64_t m, int64_t k, int64_t n, const void
   return true;
 }
 
-// split_k is reused here as an experiment knob of the forced entry point: 1 forces the
-// one-CTA form, 2 the pair form, 0 picks by shape.  No scratch is needed either way.
-GemmPlan gemm_plan(int, int64_t, int64_t m, int64_t, int64_t, int split_k) {
-  const bool pair = split_k == 2 || (split_k == 0 && m > kRowsPerCta);
-  return GemmPlan{true, pair ? 2 : 1, 0};
+// The knob of the forced entry point (its split_k argument, which this path does not need:
+// k is never split) selects the tile: knob % 16 = form (0 by shape, 1 one CTA per tile,
+// 2 a CTA pair per tile), knob / 16 = tile columns / 64 (0 by shape; 1, 2 or 4).
+// By shape: the candidate with the fewest "waves x columns" wins, a wave being one tile
+// per SM (or per pair); the one-CTA form pays a penalty because each SM then reads the
+// whole B tile from its shared memory.
+GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t, int64_t n, int knob) {
+  int form = knob % 16, tile_n = (knob / 16) * 64;
+  if (form < 0 || form > 2 || (tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) ||
+      (form == 2 && tile_n == 64))
+    return GemmPlan{false, 0, 0, 0};
+  double best = 0;
+  int best_form = 0, best_n = 0;
+  for (int f = 1; f <= 2; ++f) {
+    if (form != 0 && f != form) continue;
+    if (form == 0 && f == 2 && m <= kRowsPerCta) continue;   // a pair would idle its second CTA
+    for (int tn = 256; tn >= 64; tn >>= 1) {
+      if ((tile_n != 0 && tn != tile_n) || (f == 2 && tn == 64)) continue;
+      const int64_t tile_m = (int64_t)kRowsPerCta * f;
+      const int64_t tiles = b * ((m + tile_m - 1) / tile_m) * ((n + tn - 1) / tn);
+      const int64_t units = std::max(1, f == 2 ? sms / 2 : sms);
+      const int64_t waves = (tiles + units - 1) / units;
+      // Narrow tiles re-read A more often and amortise the epilogue hand-over worse.
+      const double cost = (double)waves * tn * (f == 1 ? 1.12 : 1.0) * (tn == 256 ? 1.0 : tn == 128 ? 1.04 : 1.10);
+      if (best_n == 0 || cost < best) { best = cost; best_form = f; best_n = tn; }
+    }
+  }
+  if (best_n == 0) return GemmPlan{false, 0, 0, 0};
+  return GemmPlan{true, best_form, best_n, 0};
 }
 
 namespace {
 
-template <bool kPair>
+template <bool kPair, int kTileN>
 cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, int64_t n,
-                        const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
-                        cudaStream_t stream) {
-  using S = Shape<kPair>;
+                        const CUtensorMap& map_a, const CUtensorMap& map_b,
+                        const CUtensorMap& map_c, float* C, cudaStream_t stream) {
+  using S = Shape<kPair, kTileN>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(gemm_kernel<kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)S::kSmemBytes);
+    attr_err = cudaFuncSetAttribute(gemm_kernel<kPair, kTileN>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::kSmemBytes);
   });
   if (attr_err != cudaSuccess) return attr_err;
 
@@ -389,7 +446,7 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   }
   cfg.attrs = attr;
   cfg.numAttrs = num_attrs;
-  return cudaLaunchKernelEx(&cfg, gemm_kernel<kPair>, map_a, map_b, p);
+  return cudaLaunchKernelEx(&cfg, gemm_kernel<kPair, kTileN>, map_a, map_b, map_c, p);
 }
 
 }  // namespace
@@ -397,11 +454,18 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m, int64_t k,
                         int64_t n, const uint16_t* A, const uint16_t* B, float* C, float*,
                         cudaStream_t stream, uint64_t* launches) {
-  CUtensorMap map_a, map_b;
-  cudaError_t e = get_maps(MapKey{A, B, b, m, k, n}, &map_a, &map_b);
+  CUtensorMap map_a, map_b, map_c;
+  cudaError_t e = get_maps(MapKey{A, B, C, b, m, k, n}, &map_a, &map_b, &map_c);
   if (e != cudaSuccess) return e;
-  e = plan.split_k == 2 ? launch_gemm<true>(dev, b, m, k, n, map_a, map_b, C, stream)
-                        : launch_gemm<false>(dev, b, m, k, n, map_a, map_b, C, stream);
+  const int code = plan.form * 1000 + plan.tile_n;
+  switch (code) {
+    case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, C, stream); break;
+    case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, stream); break;
+    case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, stream); break;
+    case 2128: e = launch_gemm<true, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, stream); break;
+    case 2256: e = launch_gemm<true, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, stream); break;
+    default: return cudaErrorInvalidValue;
+  }
   if (e == cudaSuccess) ++*launches;
   return e;
 }

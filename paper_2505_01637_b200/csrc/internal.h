@@ -47,13 +47,15 @@ cudaError_t skinny_launch(const SkinnyPlan& plan, int64_t b, int m, int64_t k, i
 // ---- tcgen05 path ------------------------------------------------------------
 struct GemmPlan {
   bool supported;
-  int split_k;
+  int form;      // 1: one CTA per 128-row tile, 2: a CTA pair per 256-row tile
+  int tile_n;    // 64, 128 or 256 columns per tile
   size_t workspace_bytes;
 };
 
 bool gemm_shape_supported(int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
                           const void* B, const void* C);
-GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int split_k);
+// `knob`: 0 = by shape; otherwise form + 16 * (tile columns / 64), either part 0 = by shape.
+GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob);
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m,
                         int64_t k, int64_t n, const uint16_t* A, const uint16_t* B, float* C,
                         float* workspace, cudaStream_t stream, uint64_t* launches);
