@@ -140,7 +140,11 @@ int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n);
 
 /*
  * Run on a given path (MORELLO_PATH_AUTO = selector) with a given split of the
- * k range across thread blocks (0 = automatic).  On the tcgen05 path, which never
+ * k range across thread blocks (0 = automatic).  On the skinny path (value % 1024) is
+ * that split and (value / 1024) picks the kernel: 0 = by shape, 1 = the register-
+ * streaming kernel (any shape), 2 = the TMA-ring GEMV kernel (m <= 4, n % 8 == 0,
+ * 16-byte-aligned B; it raises the split as needed to keep a block's k slice within
+ * 2048 rows).  On the tcgen05 path, which never
  * splits k, the argument instead selects the tile: (value % 16) is the form -- 0 = by
  * shape, 1 = one CTA per 128-row tile, 2 = a pair of CTAs per 256-row tile
  * (cta_group::2) -- and (value / 16) is the tile's column count / 64 -- 0 = by shape,
@@ -166,6 +170,13 @@ size_t morello_workspace_bytes_forced(int path, int split_k,
  * not NULL it receives the raw status word (0 when OK).
  */
 int morello_read_device_status(void* stream, uint32_t* detail);
+
+/*
+ * What the kernels size their grids by on the current device: the number of SMs and
+ * the number of two-CTA clusters (cta_group::2 pairs) the device can hold at once,
+ * which may be fewer than half the SMs.  Either pointer may be NULL.
+ */
+int morello_device_limits(int* sms, int* cta_pairs);
 
 /* Kernel launches enqueued by this library since it was loaded (all devices). */
 uint64_t morello_launch_count(void);

@@ -44,6 +44,7 @@ SIGNATURES = {
                                            _vp, _sz, _vp]),
     "morello_workspace_bytes_forced": (_sz, [_int, _int, _i64, _i64, _i64, _i64]),
     "morello_read_device_status": (_int, [_vp, ctypes.POINTER(ctypes.c_uint32)]),
+    "morello_device_limits": (_int, [ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]),
     "morello_launch_count": (ctypes.c_uint64, []),
     "morello_last_cuda_error": (_int, []),
     "morello_status_string": (ctypes.c_char_p, [_int]),
@@ -160,6 +161,13 @@ def morello_read_device_status(stream=None):
     detail = ctypes.c_uint32(0)
     st = lib().morello_read_device_status(_stream(stream), ctypes.byref(detail))
     return int(st), int(detail.value)
+
+
+def morello_device_limits():
+    """(SMs, two-CTA clusters the device holds at once) of the current device."""
+    sms, pairs = ctypes.c_int(0), ctypes.c_int(0)
+    _check(lib().morello_device_limits(ctypes.byref(sms), ctypes.byref(pairs)), "morello_device_limits")
+    return int(sms.value), int(pairs.value)
 
 
 def morello_launch_count() -> int:

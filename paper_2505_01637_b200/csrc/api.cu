@@ -94,9 +94,33 @@ int select_path(int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const
   return gemm_shape_supported(b, m, k, n, A, B, C) ? MORELLO_PATH_TCGEN05 : MORELLO_PATH_SKINNY;
 }
 
+// The knob of the forced entry point on the skinny path: knob % 1024 is the split of the k
+// range (0 = automatic), knob / 1024 picks the kernel (0 = by shape, 1 = the register-
+// streaming kernel, 2 = the TMA-ring GEMV kernel, which needs m <= 4, n % 8 == 0 and a
+// 16-byte-aligned B).
+constexpr int kKnobSplitMod = 1024;
+enum { SKINNY_AUTO = 0, SKINNY_REGISTER = 1, SKINNY_STREAM = 2 };
+
+// Which skinny kernel runs this shape: -1 = the request cannot be met.
+int skinny_kernel_for(int knob, int64_t b, int64_t m, int64_t k, int64_t n, const void* B) {
+  const int want = knob / kKnobSplitMod;
+  const bool can = m <= 4 && stream_shape_supported(b, (int)m, k, n, B) &&
+                   stream_plan(1, b, (int)m, k, n, knob % kKnobSplitMod).supported;
+  if (want == SKINNY_REGISTER) return SKINNY_REGISTER;
+  if (want == SKINNY_STREAM) return can ? SKINNY_STREAM : -1;
+  if (want != SKINNY_AUTO) return -1;
+  // Small problems finish inside one launch latency either way; the ring pays off once
+  // there is a stream of B worth pipelining.
+  return (can && k >= 256 && n >= 256) ? SKINNY_STREAM : SKINNY_REGISTER;
+}
+
 // Scratch for the skinny path over all row chunks (chunks run one after another on
 // the stream, so they share the buffer).
-size_t skinny_workspace(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int vec, int split_k) {
+size_t skinny_workspace(int sms, int64_t b, int64_t m, int64_t k, int64_t n, const void* B, int knob) {
+  const int split_k = knob % kKnobSplitMod;
+  const int which = skinny_kernel_for(knob, b, m, k, n, B);
+  if (which == SKINNY_STREAM) return stream_plan(sms, b, (int)m, k, n, split_k).workspace_bytes;
+  const int vec = skinny_vec(n, B);
   // Chunks are full (16 rows) except possibly the last one.
   const int first = (int)std::min<int64_t>(kSkinnyMaxRows, m);
   size_t need = skinny_plan(sms, b, first, k, n, vec, split_k).workspace_bytes;
@@ -106,10 +130,10 @@ size_t skinny_workspace(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int
   return need;
 }
 
-size_t workspace_for(int sms, int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n,
-                     int vec) {
-  if (path == MORELLO_PATH_TCGEN05) return gemm_plan(sms, b, m, k, n, split_k).workspace_bytes;
-  return skinny_workspace(sms, b, m, k, n, vec, split_k);
+size_t workspace_for(int sms, int path, int knob, int64_t b, int64_t m, int64_t k, int64_t n,
+                     const void* B) {
+  if (path == MORELLO_PATH_TCGEN05) return gemm_plan(sms, b, m, k, n, knob).workspace_bytes;
+  return skinny_workspace(sms, b, m, k, n, B, knob);
 }
 
 int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
@@ -139,7 +163,12 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
 
   const int sms = st->info.sms;
   const int vec = skinny_vec(n, B);
-  const size_t need = workspace_for(sms, path, split_k, b, m, k, n, vec);
+  int which = SKINNY_REGISTER;
+  if (path == MORELLO_PATH_SKINNY) {
+    which = skinny_kernel_for(split_k, b, m, k, n, B);
+    if (which < 0) return MORELLO_ERR_UNSUPPORTED_PATH;
+  }
+  const size_t need = workspace_for(sms, path, split_k, b, m, k, n, B);
   float* ws = static_cast<float*>(workspace);
   if (need > 0) {
     if (own_scratch) {
@@ -172,11 +201,16 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     if (!plan.supported) return MORELLO_ERR_UNSUPPORTED_PATH;
     e = gemm_launch(st->info, plan, b, m, k, n, static_cast<const uint16_t*>(A),
                     static_cast<const uint16_t*>(B), C, ws, s, &launches);
+  } else if (which == SKINNY_STREAM) {
+    const StreamPlan plan = stream_plan(sms, b, (int)m, k, n, split_k % kKnobSplitMod);
+    e = stream_launch(st->info, plan, b, (int)m, k, n, static_cast<const uint16_t*>(A), m * k,
+                      static_cast<const uint16_t*>(B), C, m * n, ws, s, &launches);
   } else {
     const uint16_t* a = static_cast<const uint16_t*>(A);
+    const int split = split_k % kKnobSplitMod;
     for (int64_t i0 = 0; i0 < m && e == cudaSuccess; i0 += kSkinnyMaxRows) {
       const int mc = (int)std::min<int64_t>(kSkinnyMaxRows, m - i0);
-      const SkinnyPlan plan = skinny_plan(sms, b, mc, k, n, vec, split_k);
+      const SkinnyPlan plan = skinny_plan(sms, b, mc, k, n, vec, split);
       e = skinny_launch(plan, b, mc, k, n, a + i0 * k, m * k, static_cast<const uint16_t*>(B),
                         C + i0 * n, m * n, ws, s, &launches);
     }
@@ -216,7 +250,8 @@ size_t morello_workspace_bytes_forced(int path, int split_k, int64_t b, int64_t 
   }
   if (path == MORELLO_PATH_AUTO) path = select_path(b, m, k, n, fake, fake, fake);
   if (path == MORELLO_PATH_TCGEN05 && !gemm_shape_supported(b, m, k, n, fake, fake, fake)) return 0;
-  return workspace_for(st->info.sms, path, split_k, b, m, k, n, skinny_vec(n, fake));
+  if (path == MORELLO_PATH_SKINNY && skinny_kernel_for(split_k, b, m, k, n, fake) < 0) return 0;
+  return workspace_for(st->info.sms, path, split_k, b, m, k, n, fake);
 }
 
 int morello_matmul_accum_ws(int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
@@ -308,6 +343,19 @@ int morello_read_device_status(void* stream, uint32_t* detail) {
   if ((e = cudaMemset(st->info.status, 0, 4)) != cudaSuccess) return cuda_fail(e);
   if (detail) *detail = word;
   return MORELLO_ERR_DEVICE_TIMEOUT;
+}
+
+int morello_device_limits(int* sms, int* cta_pairs) {
+  DeviceState* st = nullptr;
+  int rc;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    rc = device_state(&st);
+  }
+  if (rc != MORELLO_OK) return rc;
+  if (sms) *sms = st->info.sms;
+  if (cta_pairs) *cta_pairs = gemm_pair_units(st->info.sms);
+  return MORELLO_OK;
 }
 
 uint64_t morello_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

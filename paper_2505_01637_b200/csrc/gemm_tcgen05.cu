@@ -106,7 +106,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S::kStages; ++s) {
-      mbar_init(&bars->full[s], S::kCtas);   // one arrive.expect_tx per producer of the pair
+      mbar_init(&bars->full[s], 1);          // the (leader's) producer's arrive.expect_tx
       mbar_init(&bars->empty[s], 1);
     }
     for (int i = 0; i < 2; ++i) {
@@ -144,6 +144,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      const uint32_t leader_full = kPair ? map_to_cta(smem_u32(&bars->full[0]), 0) : 0u;
+      (void)leader_full;
       for (int64_t t = unit; t < p.tiles && ok; t += units) {
         const int mt = (int)(t % p.m_tiles);
         const int nt = (int)((t / p.m_tiles) % p.n_tiles);
@@ -155,9 +157,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           uint8_t* sa = stages + (size_t)stage * S::kStageBytes;
           uint8_t* sb = sa + kBytesA;
           if constexpr (kPair) {
-            // Both producers report to the leader's barrier: it opens once both halves landed.
-            const uint32_t full = map_to_cta(smem_u32(&bars->full[stage]), 0);
-            mbar_arrive_expect_tx_cluster(full, S::kStageBytes);
+            // Both CTAs' loads complete on the leader's barrier.  Only the leader arrives on
+            // it (a local arrive, announcing the bytes of both halves): a load of the peer
+            // that lands first just leaves the byte count negative until then, and the phase
+            // cannot end before the leader's arrival.
+            const uint32_t full = leader_full + (uint32_t)stage * 8u;
+            if (rank == 0) mbar_arrive_expect_tx(&bars->full[stage], 2 * S::kStageBytes);
             tma_load_3d_pair(sa, &map_a, full, kb * kTileK, row0, bb);
 #pragma unroll
             for (int j = 0; j < S::kBoxesB; ++j)
@@ -370,12 +375,68 @@ bool gemm_shape_supported(int64_t b, int64_t m, int64_t k, int64_t n, const void
   return true;
 }
 
+namespace {
+
+template <bool kPair, int kTileN>
+cudaError_t set_smem_attribute() {
+  static std::once_flag once;
+  static cudaError_t err = cudaSuccess;
+  std::call_once(once, [] {
+    err = cudaFuncSetAttribute(gemm_kernel<kPair, kTileN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)Shape<kPair, kTileN>::kSmemBytes);
+  });
+  return err;
+}
+
+// How many CTA pairs the device can hold at once.  A pair needs two SMs of one
+// cluster-scheduling domain, so this can be fewer than sms / 2; a persistent grid larger
+// than it would run its surplus pairs only after the first ones have finished.
+constexpr int kMaxDevices = 64;
+int g_pair_units[kMaxDevices];   // 0 = not asked yet
+std::mutex g_pair_mutex;
+
+int pair_units(int sms) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return std::max(1, sms / 2);
+  std::lock_guard<std::mutex> lock(g_pair_mutex);
+  if (g_pair_units[dev] > 0) return g_pair_units[dev];
+  int clusters = 0;
+  if (set_smem_attribute<true, 256>() == cudaSuccess) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(sms / 2 * 2), 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = Shape<true, 256>::kSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaOccupancyMaxActiveClusters(&clusters, gemm_kernel<true, 256>, &cfg) != cudaSuccess) {
+      (void)cudaGetLastError();
+      clusters = 0;
+    }
+  }
+  if (clusters <= 0) clusters = std::max(1, sms / 2 - 8);   // conservative when the query fails
+  clusters = std::min(clusters, std::max(1, sms / 2));
+  g_pair_units[dev] = clusters;
+  return clusters;
+}
+
+}  // namespace
+
+int gemm_pair_units(int sms) { return pair_units(sms); }
+
 // The knob of the forced entry point (its split_k argument, which this path does not need:
 // k is never split) selects the tile: knob % 16 = form (0 by shape, 1 one CTA per tile,
 // 2 a CTA pair per tile), knob / 16 = tile columns / 64 (0 by shape; 1, 2 or 4).
-// By shape: the candidate with the fewest "waves x columns" wins, a wave being one tile
-// per SM (or per pair); the one-CTA form pays a penalty because each SM then reads the
-// whole B tile from its shared memory.
+// By shape: with a single row of tiles (m <= 128) the call streams B once and is bound by
+// memory, so the widest tile that still gives about one thread block per SM wins.  Otherwise
+// the candidate with the fewest "waves x columns" wins, a wave being one tile per SM (or per
+// pair), weighted by what the narrower and the one-CTA tiles were measured to cost per
+// column (they re-read A more often, and a lone CTA reads the whole B tile from its own
+// shared memory).
 GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t, int64_t n, int knob) {
   int form = knob % 16, tile_n = (knob / 16) * 64;
   if (form < 0 || form > 2 || (tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) ||
@@ -383,6 +444,13 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t, int64_t n, int knob) 
     return GemmPlan{false, 0, 0, 0};
   double best = 0;
   int best_form = 0, best_n = 0;
+  if (form != 2 && tile_n == 0 && m <= kRowsPerCta) {
+    best_form = 1;
+    best_n = 64;
+    for (int tn = 256; tn >= 64; tn >>= 1)
+      if (b * ((n + tn - 1) / tn) * 5 >= (int64_t)sms * 4) { best_n = tn; break; }
+    return GemmPlan{true, best_form, best_n, 0};
+  }
   for (int f = 1; f <= 2; ++f) {
     if (form != 0 && f != form) continue;
     if (form == 0 && f == 2 && m <= kRowsPerCta) continue;   // a pair would idle its second CTA
@@ -390,10 +458,10 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t, int64_t n, int knob) 
       if ((tile_n != 0 && tn != tile_n) || (f == 2 && tn == 64)) continue;
       const int64_t tile_m = (int64_t)kRowsPerCta * f;
       const int64_t tiles = b * ((m + tile_m - 1) / tile_m) * ((n + tn - 1) / tn);
-      const int64_t units = std::max(1, f == 2 ? sms / 2 : sms);
+      const int64_t units = std::max(1, f == 2 ? pair_units(sms) : sms);
       const int64_t waves = (tiles + units - 1) / units;
-      // Narrow tiles re-read A more often and amortise the epilogue hand-over worse.
-      const double cost = (double)waves * tn * (f == 1 ? 1.12 : 1.0) * (tn == 256 ? 1.0 : tn == 128 ? 1.04 : 1.10);
+      const double cost = (double)waves * tn * (f == 1 ? 1.15 : 1.0) *
+                          (tn == 256 ? 1.0 : tn == 128 ? 1.25 : 1.6);
       if (best_n == 0 || cost < best) { best = cost; best_form = f; best_n = tn; }
     }
   }
@@ -408,12 +476,7 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
                         const CUtensorMap& map_a, const CUtensorMap& map_b,
                         const CUtensorMap& map_c, float* C, cudaStream_t stream) {
   using S = Shape<kPair, kTileN>;
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(gemm_kernel<kPair, kTileN>,
-                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::kSmemBytes);
-  });
+  const cudaError_t attr_err = set_smem_attribute<kPair, kTileN>();
   if (attr_err != cudaSuccess) return attr_err;
 
   GemmParams p{};
@@ -426,7 +489,7 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   p.k_blocks = (int)((k + kTileK - 1) / kTileK);
   p.status = dev.status;
 
-  const int64_t max_units = kPair ? dev.sms / 2 : dev.sms;
+  const int64_t max_units = kPair ? pair_units(dev.sms) : dev.sms;
   const int64_t units = std::min<int64_t>(p.tiles, max_units);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(units * S::kCtas), 1, 1);

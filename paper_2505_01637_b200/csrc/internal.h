@@ -44,6 +44,29 @@ cudaError_t skinny_launch(const SkinnyPlan& plan, int64_t b, int m, int64_t k, i
                           int64_t c_batch, float* workspace, cudaStream_t stream,
                           uint64_t* launches);
 
+// Enqueues the slice-ordered reduce: C[b, i, :] += partial[0] + partial[1] + ... for the
+// b * m * n sums of one row chunk (partial is [split_k][b][m][n], c_batch the batch stride of C).
+cudaError_t skinny_reduce_launch(const float* partial, float* C, int64_t b, int m, int64_t n,
+                                 int64_t c_batch, int split_k, cudaStream_t stream);
+
+// ---- streaming GEMV (FP32 FMA, B through a TMA ring, m <= 4) ------------------
+struct StreamPlan {
+  bool supported;
+  int m_tile;        // 1, 2 or 4
+  int strips;        // thread blocks along n (64 columns each)
+  int split_k;       // thread blocks along k
+  int k_per_split;   // multiple of 64
+  size_t smem_bytes;
+  size_t workspace_bytes;  // partial sums [split_k][b][m][n] f32 when split_k > 1
+};
+// Needs n % 8 == 0 and a 16-byte-aligned B (the TMA engine addresses B through a tensor map).
+bool stream_shape_supported(int64_t b, int m, int64_t k, int64_t n, const void* B);
+StreamPlan stream_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int split_k);
+cudaError_t stream_launch(const DeviceInfo& dev, const StreamPlan& plan, int64_t b, int m, int64_t k,
+                          int64_t n, const uint16_t* A, int64_t a_batch, const uint16_t* B, float* C,
+                          int64_t c_batch, float* workspace, cudaStream_t stream,
+                          uint64_t* launches);
+
 // ---- tcgen05 path ------------------------------------------------------------
 struct GemmPlan {
   bool supported;
@@ -56,6 +79,8 @@ bool gemm_shape_supported(int64_t b, int64_t m, int64_t k, int64_t n, const void
                           const void* B, const void* C);
 // `knob`: 0 = by shape; otherwise form + 16 * (tile columns / 64), either part 0 = by shape.
 GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob);
+// CTA pairs (cta_group::2) the current device can hold at once.
+int gemm_pair_units(int sms);
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m,
                         int64_t k, int64_t n, const uint16_t* A, const uint16_t* B, float* C,
                         float* workspace, cudaStream_t stream, uint64_t* launches);

@@ -378,15 +378,19 @@ cudaError_t skinny_launch(const SkinnyPlan& plan, int64_t b, int m, int64_t k, i
     ++*launches;
   }
   if (plan.split_k > 1) {
-    const int64_t total = b * m * n;
-    const int64_t blocks = (total + 255) / 256;
-    cudaError_t e = launch_pdl(reduce_kernel, dim3((unsigned)blocks, 1, 1), 256, 0, stream,
-                               (const float*)workspace, C, total, (int64_t)m * n, c_batch,
-                               plan.split_k);
+    cudaError_t e = skinny_reduce_launch(workspace, C, b, m, n, c_batch, plan.split_k, stream);
     if (e != cudaSuccess) return e;
     ++*launches;
   }
   return cudaSuccess;
+}
+
+cudaError_t skinny_reduce_launch(const float* partial, float* C, int64_t b, int m, int64_t n,
+                                 int64_t c_batch, int split_k, cudaStream_t stream) {
+  const int64_t total = b * m * n;
+  const int64_t blocks = (total + 255) / 256;
+  return launch_pdl(reduce_kernel, dim3((unsigned)blocks, 1, 1), 256, 0, stream, partial, C, total,
+                    (int64_t)m * n, c_batch, split_k);
 }
 
 }  // namespace morello

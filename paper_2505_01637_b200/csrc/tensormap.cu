@@ -23,7 +23,8 @@ void resolve() {
 
 cudaError_t make_tensor_map_3d(CUtensorMap* out, CUtensorMapDataType dtype, int elem_bytes,
                                const void* base, uint64_t d0, uint64_t d1, uint64_t d2,
-                               uint32_t box0, uint32_t box1, CUtensorMapSwizzle swizzle) {
+                               uint32_t box0, uint32_t box1, CUtensorMapSwizzle swizzle,
+                               CUtensorMapL2promotion promotion) {
   std::call_once(g_once, resolve);
   if (!g_encode) return cudaErrorNotSupported;
   cuuint64_t dims[3] = {d0, d1, d2};
@@ -31,7 +32,7 @@ cudaError_t make_tensor_map_3d(CUtensorMap* out, CUtensorMapDataType dtype, int 
   cuuint32_t box[3] = {box0, box1, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = g_encode(out, dtype, 3, const_cast<void*>(base), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, promotion,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }

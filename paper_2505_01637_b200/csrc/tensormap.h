@@ -14,6 +14,7 @@ namespace morello {
 // multiple of 16, box0 * elem_bytes <= the swizzle span.
 cudaError_t make_tensor_map_3d(CUtensorMap* out, CUtensorMapDataType dtype, int elem_bytes,
                                const void* base, uint64_t d0, uint64_t d1, uint64_t d2,
-                               uint32_t box0, uint32_t box1, CUtensorMapSwizzle swizzle);
+                               uint32_t box0, uint32_t box1, CUtensorMapSwizzle swizzle,
+                               CUtensorMapL2promotion promotion = CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 
 }  // namespace morello

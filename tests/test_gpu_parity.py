@@ -112,6 +112,66 @@ def test_caller_workspace_and_its_size_check():
     assert torch.equal(before, dC)
 
 
+# ------------------------------------- T3b: the TMA-ring GEMV kernel, forced (knob 2048 + split)
+STREAM = 2 * 1024
+
+
+@pytest.mark.parametrize("shape", [
+    (1, 1, 64, 64),          # one box
+    (1, 1, 2048, 16384),     # the headline shape
+    (1, 1, 100, 72),         # ragged k (scalar staging of A) and a partial last strip
+    (2, 3, 1000, 200),       # batches, m = 3 in the 4-row kernel, k % 8 == 0 but ragged boxes
+    (3, 2, 321, 136),
+    (1, 4, 5000, 328),       # k longer than one block's slice: the planner splits k
+    (1, 4, 2048, 4096),
+    (2, 1, 8192, 64),        # few strips, long k
+])
+def test_stream_kernel_matches_oracle(shape):
+    b, m, k, n = shape
+    A, B, C = w.make(b, m, k, n, seed=sum(shape), ab="int4", c="normal")
+    check_full(A, B, C, integer=True, path=mb.MORELLO_PATH_SKINNY, split_k=STREAM, what="stream %s" % (shape,))
+    A, B, C = w.make(b, m, k, n, seed=sum(shape) + 1, ab="uniform", c="normal")
+    check_full(A, B, C, integer=False, path=mb.MORELLO_PATH_SKINNY, split_k=STREAM, what="stream %s" % (shape,))
+
+
+@pytest.mark.parametrize("split_k", [1, 2, 3, 7, 32])
+def test_stream_kernel_forced_splits(split_k):
+    for (b, m, k, n) in [(1, 1, 2048, 256), (2, 3, 1000, 72), (1, 4, 4096, 64)]:
+        A, B, C = w.make(b, m, k, n, seed=split_k, ab="int4", c="normal")
+        check_full(A, B, C, integer=True, path=mb.MORELLO_PATH_SKINNY, split_k=STREAM + split_k,
+                   what="stream split %d %s" % (split_k, (b, m, k, n)))
+
+
+def test_stream_kernel_one_hot_and_repeatability():
+    b, m, k, n = 2, 2, 192, 136
+    rng = np.random.default_rng(3)
+    Bv = rng.integers(-100, 101, size=(b, k, n)).astype(np.float32)
+    C = rng.integers(-50, 51, size=(b, m, n)).astype(np.float32)
+    for (b0, i0, p0) in [(0, 0, 0), (1, 1, 191), (0, 1, 64)]:
+        A1 = np.zeros((b, m, k), np.float32)
+        A1[b0, i0, p0] = 2.0
+        want = C.copy()
+        want[b0, i0, :] += 2.0 * Bv[b0, p0, :]
+        got = gpu_run(w.f32_to_bf16_rne(A1), w.f32_to_bf16_rne(Bv), C, path=mb.MORELLO_PATH_SKINNY, split_k=STREAM)
+        assert_bit_exact(got, want, "stream one-hot A at %s" % ((b0, i0, p0),))
+    A, B, C = w.make(1, 1, 2048, 16384, seed=21, ab="uniform", c="normal")
+    first = gpu_run(A, B, C, path=mb.MORELLO_PATH_SKINNY, split_k=STREAM)
+    for _ in range(3):
+        assert np.array_equal(bits(gpu_run(A, B, C, path=mb.MORELLO_PATH_SKINNY, split_k=STREAM)), bits(first))
+
+
+def test_stream_kernel_refuses_what_it_cannot_address():
+    b, m, k, n = 1, 2, 64, 36             # n not a multiple of 8
+    dA, dB, dC = to_dev(*w.make(b, m, k, n, seed=13))
+    with pytest.raises(mb.MorelloError) as e:
+        mb.morello_matmul_accum_forced(mb.MORELLO_PATH_SKINNY, STREAM, b, m, k, n, dA, dB, dC)
+    assert e.value.status == mb.MORELLO_ERR_UNSUPPORTED_PATH
+    dA, dB, dC = to_dev(*w.make(1, 5, 64, 64, seed=13))      # more than 4 rows
+    with pytest.raises(mb.MorelloError) as e:
+        mb.morello_matmul_accum_forced(mb.MORELLO_PATH_SKINNY, STREAM, 1, 5, 64, 64, dA, dB, dC)
+    assert e.value.status == mb.MORELLO_ERR_UNSUPPORTED_PATH
+
+
 # ------------------------------------------------------------- T4: determinism
 @pytest.mark.parametrize("shape", [(1, 1, 2048, 16384), (1, 16, 2048, 1024), (1, 3, 8192, 64)])
 def test_repeated_calls_give_identical_bits(shape):
