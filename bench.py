@@ -422,10 +422,12 @@ def run_ours(args):
                 continue
             iters, wu = plan[idx]
             extra.append(bench_config(torch, mb, idx, iters, wu, peaks, windows))
-            if idx == 2 and mb.morello_select_path(*w.CONFIGS[2].shape) == mb.MORELLO_PATH_SKINNY:
-                try:                            # crossover config: also on the tensor-core path
-                    extra.append(bench_config(torch, mb, idx, iters, wu, peaks, windows,
-                                              path=mb.MORELLO_PATH_TCGEN05))
+            if idx == 2:                        # crossover config: also on the path not chosen
+                other = (mb.MORELLO_PATH_TCGEN05
+                         if mb.morello_select_path(*w.CONFIGS[2].shape) == mb.MORELLO_PATH_SKINNY
+                         else mb.MORELLO_PATH_SKINNY)
+                try:
+                    extra.append(bench_config(torch, mb, idx, 100, wu, peaks, windows, path=other))
                 except mb.MorelloError:
                     pass
     sampler.stop()
@@ -455,7 +457,7 @@ def run_ours(args):
             "roofline": {"bound": "hbm", "achieved": per_launch_gbs, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": per_launch_gbs / peaks["hbm_gbs"],
                          "peak_kind": peak_kind, "frac_of_nominal_8TBs": per_launch_gbs / NOMINAL_HBM_GBS,
-                         "traffic": traffic.get(cfg.name), "kernel": "skinny_kernel<1,8>"},
+                         "traffic": traffic.get(cfg.name), "kernel": "gemv_stream_kernel<1>"},
             "graph_replay_us_per_call": graph_us,
             "cpu_baseline": cpu,
             "configs": extra,

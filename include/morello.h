@@ -135,7 +135,11 @@ size_t morello_noalloc_scratch_limit(void);
 /* --- introspection and experiments (tests and benchmarks) ------------------ */
 
 /* The path the selector picks for this shape with 16-byte-aligned operands:
- * MORELLO_PATH_SKINNY or MORELLO_PATH_TCGEN05 (-1 for an invalid shape). */
+ * MORELLO_PATH_SKINNY or MORELLO_PATH_TCGEN05 (-1 for an invalid shape).  Up to 4 rows
+ * go to the FP32-FMA kernels; from 5 rows on the tcgen05 kernel runs whenever it can
+ * address the shape (k % 8 == 0, n % 8 == 0) and, up to 16 rows, B has enough columns
+ * to give half the SMs a tile (the choice uses the current device's SM count, 148 when
+ * no device is usable). */
 int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n);
 
 /*
@@ -143,8 +147,8 @@ int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n);
  * k range across thread blocks (0 = automatic).  On the skinny path (value % 1024) is
  * that split and (value / 1024) picks the kernel: 0 = by shape, 1 = the register-
  * streaming kernel (any shape), 2 = the TMA-ring GEMV kernel (m <= 4, n % 8 == 0,
- * 16-byte-aligned B; it raises the split as needed to keep a block's k slice within
- * 2048 rows).  On the tcgen05 path, which never
+ * 16-byte-aligned B; it raises the split as needed to keep the part of A a block
+ * stages within 32 KiB: 16384 / m rows of k per block, m rounded up to 1, 2 or 4).  On the tcgen05 path, which never
  * splits k, the argument instead selects the tile: (value % 16) is the form -- 0 = by
  * shape, 1 = one CTA per 128-row tile, 2 = a pair of CTAs per 256-row tile
  * (cta_group::2) -- and (value / 16) is the tile's column count / 64 -- 0 = by shape,

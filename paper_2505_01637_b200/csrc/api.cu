@@ -88,10 +88,19 @@ int validate(int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const vo
   return MORELLO_OK;
 }
 
-int select_path(int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const void* B,
+// Measured on the 2048 x 16384 weight shape: the FP32-FMA kernels win up to 4 rows (11 us at
+// m = 1, 16.6 us at m = 4, against 20 us on the tensor path) and lose from 5 rows on (35 us at
+// m = 8, 85 us at m = 16, against 19 us), because every extra row costs them one FMA per
+// element of B while the tensor cores take up to 128 rows for the price of one.  Between 5
+// and 16 rows the tensor path still needs enough column tiles to occupy the device; a tall
+// and narrow B (few columns, long k) is better served by the FMA kernel's split of k.
+constexpr int kFmaMaxRows = 4;
+int select_path(int sms, int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const void* B,
                 const void* C) {
-  if (m <= kSkinnyMaxRows) return MORELLO_PATH_SKINNY;
-  return gemm_shape_supported(b, m, k, n, A, B, C) ? MORELLO_PATH_TCGEN05 : MORELLO_PATH_SKINNY;
+  if (m <= kFmaMaxRows) return MORELLO_PATH_SKINNY;
+  if (!gemm_shape_supported(b, m, k, n, A, B, C)) return MORELLO_PATH_SKINNY;
+  if (m <= kSkinnyMaxRows && b * ((n + 63) / 64) * 2 < sms) return MORELLO_PATH_SKINNY;
+  return MORELLO_PATH_TCGEN05;
 }
 
 // The knob of the forced entry point on the skinny path: knob % 1024 is the split of the k
@@ -154,7 +163,7 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
   if (empty) return MORELLO_OK;
 
   if (path == MORELLO_PATH_AUTO) {
-    path = select_path(b, m, k, n, A, B, C);
+    path = select_path(st->info.sms, b, m, k, n, A, B, C);
   } else if (path == MORELLO_PATH_TCGEN05) {
     if (!gemm_shape_supported(b, m, k, n, A, B, C)) return MORELLO_ERR_UNSUPPORTED_PATH;
   } else if (path != MORELLO_PATH_SKINNY) {
@@ -248,7 +257,7 @@ size_t morello_workspace_bytes_forced(int path, int split_k, int64_t b, int64_t 
     std::lock_guard<std::mutex> lock(g_mutex);
     if (device_state(&st) != MORELLO_OK) return 0;
   }
-  if (path == MORELLO_PATH_AUTO) path = select_path(b, m, k, n, fake, fake, fake);
+  if (path == MORELLO_PATH_AUTO) path = select_path(st->info.sms, b, m, k, n, fake, fake, fake);
   if (path == MORELLO_PATH_TCGEN05 && !gemm_shape_supported(b, m, k, n, fake, fake, fake)) return 0;
   if (path == MORELLO_PATH_SKINNY && skinny_kernel_for(split_k, b, m, k, n, fake) < 0) return 0;
   return workspace_for(st->info.sms, path, split_k, b, m, k, n, fake);
@@ -321,7 +330,14 @@ int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n) {
   bool empty = false;
   const void* fake = reinterpret_cast<const void*>(uintptr_t(4096));
   if (validate(b, m, k, n, fake, fake, fake, &empty) != MORELLO_OK) return -1;
-  return select_path(b, m, k, n, fake, fake, fake);
+  // The choice depends on the SM count; without a usable device, a B200's is assumed.
+  int sms = 148;
+  DeviceState* st = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (device_state(&st) == MORELLO_OK) sms = st->info.sms;
+  }
+  return select_path(sms, b, m, k, n, fake, fake, fake);
 }
 
 int morello_read_device_status(void* stream, uint32_t* detail) {

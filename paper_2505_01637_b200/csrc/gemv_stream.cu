@@ -46,10 +46,10 @@ using namespace sm100;
 #define MORELLO_GEMV_STRIP_COLS 64
 #endif
 #ifndef MORELLO_GEMV_STAGES
-#define MORELLO_GEMV_STAGES 6
+#define MORELLO_GEMV_STAGES 10
 #endif
 #ifndef MORELLO_GEMV_PREFETCH_BOXES
-#define MORELLO_GEMV_PREFETCH_BOXES 16
+#define MORELLO_GEMV_PREFETCH_BOXES 12
 #endif
 constexpr int kStripCols = MORELLO_GEMV_STRIP_COLS;         // columns per thread block: 64 or 128
 constexpr int kBoxRows = 64;                                // k rows per stage
@@ -58,7 +58,8 @@ constexpr int kStages = MORELLO_GEMV_STAGES;
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumers = 32 * kConsumerWarps;
 constexpr int kThreads = 32 + kConsumers;
-constexpr int kMaxSliceK = 2048;                            // rows of A staged per block
+constexpr int kMaxSliceBytes = 32 * 1024;                   // bf16 rows of A staged per block
+constexpr int max_slice_k(int m_tile) { return kMaxSliceBytes / (2 * m_tile); }
 constexpr int kPrefetchBoxes = MORELLO_GEMV_PREFETCH_BOXES; // boxes asked into L2 before the wait
 constexpr int kLanesPerRow = kStripCols / 8;                // 16-byte chunks per box row
 constexpr int kRowsPerWarp = 32 / kLanesPerRow;             // box rows one warp-wide load covers
@@ -346,7 +347,7 @@ cudaError_t launch(const StreamPlan& plan, const CUtensorMap& map, const StreamP
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [&] {
     attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)smem_for(M_T, kMaxSliceK));
+                                    (int)smem_for(M_T, max_slice_k(M_T)));
   });
   if (attr_err != cudaSuccess) return attr_err;
   cudaLaunchConfig_t cfg{};
@@ -382,13 +383,14 @@ StreamPlan stream_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int spli
     s = 1;
     if (blocks * 10 < (int64_t)sms * 13) s = std::min<int64_t>((2 * sms + blocks - 1) / blocks, k / 512);
   }
-  s = std::max<int64_t>(s, (k + kMaxSliceK - 1) / kMaxSliceK);
+  const int slice_cap = max_slice_k(pl.m_tile);
+  s = std::max<int64_t>(s, (k + slice_cap - 1) / slice_cap);
   s = std::max<int64_t>(1, std::min<int64_t>(s, (k + kBoxRows - 1) / kBoxRows));
   int64_t kps = (k + s - 1) / s;
   kps = (kps + kBoxRows - 1) / kBoxRows * kBoxRows;
   pl.k_per_split = (int)kps;
   pl.split_k = (int)((k + kps - 1) / kps);
-  pl.supported = kps <= kMaxSliceK;
+  pl.supported = kps <= slice_cap;
   pl.smem_bytes = smem_for(pl.m_tile, pl.k_per_split);
   pl.workspace_bytes = pl.split_k > 1 ? (size_t)pl.split_k * b * m * n * 4 : 0;
   return pl;
