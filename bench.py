@@ -55,12 +55,27 @@ def load_peaks():
 
 
 def load_traffic():
-    """DRAM bytes per launch from the committed ncu summaries (None if absent)."""
-    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    """DRAM bytes per launch from the committed ncu summaries (profiles/dram_traffic.txt).
+    A figure counts only while the kernel's source file still has the hash it had when
+    the counters were taken; otherwise the entry is dropped (reported as null)."""
+    import hashlib
+    out = {}
     try:
-        return json.load(open(path))
-    except Exception:
-        return {}
+        lines = open(os.path.join(ROOT, "profiles", "dram_traffic.txt")).read().splitlines()
+    except OSError:
+        return out
+    for line in lines:
+        parts = line.split()
+        if len(parts) != 4 or line.startswith("#"):
+            continue
+        name, nbytes, src, digest = parts
+        try:
+            blob = open(os.path.join(ROOT, "paper_2505_01637_b200", "csrc", src), "rb").read()
+        except OSError:
+            continue
+        if hashlib.sha256(blob).hexdigest().startswith(digest):
+            out[name] = int(nbytes)
+    return out
 
 
 # ------------------------------------------------------------------ clock sampler
