@@ -64,6 +64,12 @@ struct Shape {
   static_assert(kColsB % 64 == 0 && kTileN <= kAccStride, "tile shape");
 };
 
+// Height of the TMA box of A: a whole 128-row tile, or, when the matrix has fewer rows than
+// that (then there is one row of tiles, in the one-CTA form), m rounded up to a multiple of 16.
+inline int a_box_rows(int64_t m) {
+  return m >= kRowsPerCta ? kRowsPerCta : (int)((m + 15) / 16 * 16);
+}
+
 struct GemmParams {
   float* C;
   int64_t m, n, k;
@@ -72,6 +78,7 @@ struct GemmParams {
   int64_t tiles;    // b * m_tiles * n_tiles
   int k_blocks;
   uint32_t* status;
+  int a_box_rows;  // rows of A one TMA box brings: 128, or m rounded up to 16 when m < 128
 };
 
 struct Barriers {
@@ -119,6 +126,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     tma_prefetch_descriptor(&map_b);
     tma_prefetch_descriptor(&map_c);
   }
+  if (p.a_box_rows < kRowsPerCta) {
+    // Few rows: the TMA box of A is only as high as m needs (a box that is mostly outside the
+    // tensor loads several times slower than its in-bounds part alone).  The rows of the stage
+    // the box never writes are zeroed once, here; the MMA reads them as zeros.
+    for (int s2 = 0; s2 < S::kStages; ++s2) {
+      uint4* z = reinterpret_cast<uint4*>(stages + (size_t)s2 * S::kStageBytes);
+      for (int q = threadIdx.x; q < kBytesA / 16; q += kThreads) z[q] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    fence_proxy_async_smem();
+  }
   if (warp == 1) {
     if constexpr (kPair) {
       tmem_alloc_pair(&bars->tmem_base, kTmemColumns);
@@ -162,13 +179,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             // that lands first just leaves the byte count negative until then, and the phase
             // cannot end before the leader's arrival.
             const uint32_t full = leader_full + (uint32_t)stage * 8u;
-            if (rank == 0) mbar_arrive_expect_tx(&bars->full[stage], 2 * S::kStageBytes);
+            if (rank == 0)
+              mbar_arrive_expect_tx(&bars->full[stage], 2 * (S::kBytesB + p.a_box_rows * (kTileK * 2)));
             tma_load_3d_pair(sa, &map_a, full, kb * kTileK, row0, bb);
 #pragma unroll
             for (int j = 0; j < S::kBoxesB; ++j)
               tma_load_3d_pair(sb + j * kBoxBytesB, &map_b, full, col0 + j * 64, kb * kTileK, bb);
           } else {
-            mbar_arrive_expect_tx(&bars->full[stage], S::kStageBytes);
+            mbar_arrive_expect_tx(&bars->full[stage], S::kBytesB + p.a_box_rows * (kTileK * 2));
             tma_load_3d(sa, &map_a, &bars->full[stage], kb * kTileK, row0, bb);
 #pragma unroll
             for (int j = 0; j < S::kBoxesB; ++j)
@@ -342,7 +360,7 @@ cudaError_t get_maps(const MapKey& key, CUtensorMap* ma, CUtensorMap* mb, CUtens
   e.key = key;
   cudaError_t err = make_tensor_map_3d(&e.map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, key.a,
                                        (uint64_t)key.k, (uint64_t)key.m, (uint64_t)key.bsz, kTileK,
-                                       kRowsPerCta, CU_TENSOR_MAP_SWIZZLE_128B);
+                                       (uint32_t)a_box_rows(key.m), CU_TENSOR_MAP_SWIZZLE_128B);
   if (err != cudaSuccess) return err;
   err = make_tensor_map_3d(&e.map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, key.b, (uint64_t)key.n,
                            (uint64_t)key.k, (uint64_t)key.bsz, 64, kTileK,
@@ -488,6 +506,7 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   p.tiles = b * p.m_tiles * (int64_t)p.n_tiles;
   p.k_blocks = (int)((k + kTileK - 1) / kTileK);
   p.status = dev.status;
+  p.a_box_rows = a_box_rows(m);
 
   const int64_t max_units = kPair ? pair_units(dev.sms) : dev.sms;
   const int64_t units = std::min<int64_t>(p.tiles, max_units);
