@@ -76,6 +76,8 @@ struct GemmParams {
   int64_t c_batch;  // m * n
   int m_tiles, n_tiles;
   int64_t tiles;    // b * m_tiles * n_tiles
+  int64_t whole;    // work items [0, whole) are whole tiles, in tile order;
+  int64_t items;    // items [whole, items) are the column halves of tiles [whole, tiles)
   int k_blocks;
   uint32_t* status;
   int a_box_rows;  // rows of A one TMA box brings: 128, or m rounded up to 16 when m < 128
@@ -89,6 +91,30 @@ struct Barriers {
   uint32_t tmem_base;
   int abort_flag;
 };
+
+// One unit of work of a thread block (or pair): a tile, or the left / right column half of one.
+struct Item {
+  int mt, nt, bb;
+  int n_off;   // first column of the item inside its tile
+  int cols;    // columns of the item: the tile's width or half of it
+};
+template <int kTileN>
+__device__ __forceinline__ Item decode_item(const GemmParams& p, int64_t t) {
+  Item it;
+  int64_t tile = t;
+  it.n_off = 0;
+  it.cols = kTileN;
+  if (t >= p.whole) {
+    const int64_t h = t - p.whole;
+    tile = p.whole + (h >> 1);
+    it.cols = kTileN / 2;
+    it.n_off = (int)(h & 1) * (kTileN / 2);
+  }
+  it.mt = (int)(tile % p.m_tiles);
+  it.nt = (int)((tile / p.m_tiles) % p.n_tiles);
+  it.bb = (int)(tile / ((int64_t)p.m_tiles * p.n_tiles));
+  return it;
+}
 
 template <bool kPair, int kTileN>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -163,12 +189,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       bool ok = true;
       const uint32_t leader_full = kPair ? map_to_cta(smem_u32(&bars->full[0]), 0) : 0u;
       (void)leader_full;
-      for (int64_t t = unit; t < p.tiles && ok; t += units) {
-        const int mt = (int)(t % p.m_tiles);
-        const int nt = (int)((t / p.m_tiles) % p.n_tiles);
-        const int bb = (int)(t / ((int64_t)p.m_tiles * p.n_tiles));
-        const int row0 = mt * S::kTileM + (int)rank * kRowsPerCta;
-        const int col0 = nt * kTileN + (int)rank * S::kColsB;
+      for (int64_t t = unit; t < p.items && ok; t += units) {
+        const Item it = decode_item<kTileN>(p, t);
+        const int bb = it.bb;
+        const int row0 = it.mt * S::kTileM + (int)rank * kRowsPerCta;
+        const int cols_b = it.cols / S::kCtas;            // columns of B this CTA brings
+        const int boxes_b = cols_b / 64;
+        const int col0 = it.nt * kTileN + it.n_off + (int)rank * cols_b;
+        const uint32_t stage_tx = (uint32_t)(boxes_b * kBoxBytesB + p.a_box_rows * (kTileK * 2));
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!(ok = mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag, p.status, 1))) break;
           uint8_t* sa = stages + (size_t)stage * S::kStageBytes;
@@ -180,18 +208,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             // cannot end before the leader's arrival.
             const uint32_t full = leader_full + (uint32_t)stage * 8u;
             if (rank == 0)
-              mbar_arrive_expect_tx(&bars->full[stage], 2 * (S::kBytesB + p.a_box_rows * (kTileK * 2)));
+              mbar_arrive_expect_tx(&bars->full[stage], 2 * stage_tx);
             tma_load_3d_pair(sa, &map_a, full, kb * kTileK, row0, bb);
 #pragma unroll
             for (int j = 0; j < S::kBoxesB; ++j)
-              tma_load_3d_pair(sb + j * kBoxBytesB, &map_b, full, col0 + j * 64, kb * kTileK, bb);
+              if (j < boxes_b)
+                tma_load_3d_pair(sb + j * kBoxBytesB, &map_b, full, col0 + j * 64, kb * kTileK, bb);
           } else {
-            mbar_arrive_expect_tx(&bars->full[stage], S::kBytesB + p.a_box_rows * (kTileK * 2));
+            mbar_arrive_expect_tx(&bars->full[stage], stage_tx);
             tma_load_3d(sa, &map_a, &bars->full[stage], kb * kTileK, row0, bb);
 #pragma unroll
             for (int j = 0; j < S::kBoxesB; ++j)
-              tma_load_3d(sb + j * kBoxBytesB, &map_b, &bars->full[stage], col0 + j * 64,
-                          kb * kTileK, bb);
+              if (j < boxes_b)
+                tma_load_3d(sb + j * kBoxBytesB, &map_b, &bars->full[stage], col0 + j * 64,
+                            kb * kTileK, bb);
           }
           if (++stage == S::kStages) { stage = 0; phase ^= 1; }
         }
@@ -200,13 +230,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (rank == 0 && elect_one()) {
-      constexpr uint32_t idesc = instr_desc_bf16(S::kTileM, kTileN, false, true);
+      constexpr uint32_t idesc_tile = instr_desc_bf16(S::kTileM, kTileN, false, true);
+      constexpr uint32_t idesc_half = instr_desc_bf16(S::kTileM, kTileN / 2, false, true);
       int stage = 0;
       uint32_t phase = 0;
       int buf = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int64_t t = unit; t < p.tiles && ok; t += units) {
+      for (int64_t t = unit; t < p.items && ok; t += units) {
+        const uint32_t idesc = t < p.whole ? idesc_tile : idesc_half;
         if (!(ok = mbar_wait(&bars->acc_empty[buf], acc_phase ^ 1, abort_flag, p.status, 2))) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + (uint32_t)buf * kAccStride;
@@ -249,20 +281,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     uint32_t acc_phase = 0;
     uint32_t blk = 0;              // alternates between this warp's two blocks
     bool ok = true;
-    for (int64_t t = unit; t < p.tiles && ok; t += units) {
-      const int mt = (int)(t % p.m_tiles);
-      const int nt = (int)((t / p.m_tiles) % p.n_tiles);
-      const int bb = (int)(t / ((int64_t)p.m_tiles * p.n_tiles));
+    for (int64_t t = unit; t < p.items && ok; t += units) {
+      const Item it = decode_item<kTileN>(p, t);
+      const int mt = it.mt;
+      const int bb = it.bb;
       ok = mbar_wait(&bars->acc_full[buf], acc_phase, abort_flag, p.status, 4);
       ok = __all_sync(0xffffffffu, ok);  // also reconverges the warp for the aligned TMEM loads
       if (!ok) break;
       tc_fence_after_sync();
       const int row0 = mt * S::kTileM + (int)rank * kRowsPerCta + quarter * 32;
-      const int col0 = nt * kTileN;
+      const int col0 = it.nt * kTileN + it.n_off;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * kAccStride;
       const bool rows_live = row0 < p.m;   // warp-uniform
 #pragma unroll 1
-      for (int c = 0; c < kTileN; c += kEpiCols) {
+      for (int c = 0; c < it.cols; c += kEpiCols) {
         const bool live = rows_live && (col0 + c < p.n);
         uint32_t r[32];
         if (live) {
@@ -272,7 +304,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           tmem_ld_32x32(taddr + c, r);
           tmem_ld_wait();
         }
-        if (c + kEpiCols == kTileN) {
+        if (c + kEpiCols == it.cols) {
           // The accumulator has left tensor memory: hand the buffer back to the MMA issuer.
           tc_fence_before_sync();
           __syncwarp();
@@ -456,10 +488,12 @@ int gemm_pair_units(int sms) { return pair_units(sms); }
 // column (they re-read A more often, and a lone CTA reads the whole B tile from its own
 // shared memory).
 GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t, int64_t n, int knob) {
+  const bool halves = (knob / 256) == 0;
+  knob %= 256;
   int form = knob % 16, tile_n = (knob / 16) * 64;
   if (form < 0 || form > 2 || (tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) ||
       (form == 2 && tile_n == 64))
-    return GemmPlan{false, 0, 0, 0};
+    return GemmPlan{false, 0, 0, 0, false};
   double best = 0;
   int best_form = 0, best_n = 0;
   if (form != 2 && tile_n == 0 && m <= kRowsPerCta) {
@@ -467,7 +501,7 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t, int64_t n, int knob) 
     best_n = 64;
     for (int tn = 256; tn >= 64; tn >>= 1)
       if (b * ((n + tn - 1) / tn) * 5 >= (int64_t)sms * 4) { best_n = tn; break; }
-    return GemmPlan{true, best_form, best_n, 0};
+    return GemmPlan{true, best_form, best_n, 0, halves};
   }
   for (int f = 1; f <= 2; ++f) {
     if (form != 0 && f != form) continue;
@@ -477,14 +511,18 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t, int64_t n, int knob) 
       const int64_t tile_m = (int64_t)kRowsPerCta * f;
       const int64_t tiles = b * ((m + tile_m - 1) / tile_m) * ((n + tn - 1) / tn);
       const int64_t units = std::max(1, f == 2 ? pair_units(sms) : sms);
-      const int64_t waves = (tiles + units - 1) / units;
+      const int64_t tail = tiles % units;
+      const bool cut = halves && tiles > units && tail > 0 && 2 * tail <= units &&
+                       (tn / f / 2) % 64 == 0;
+      // A last wave cut into halves costs about 0.6 of a whole one.
+      const double waves = (double)(tiles / units) + (tail == 0 ? 0.0 : cut ? 0.625 : 1.0);
       const double cost = (double)waves * tn * (f == 1 ? 1.15 : 1.0) *
                           (tn == 256 ? 1.0 : tn == 128 ? 1.25 : 1.6);
       if (best_n == 0 || cost < best) { best = cost; best_form = f; best_n = tn; }
     }
   }
-  if (best_n == 0) return GemmPlan{false, 0, 0, 0};
-  return GemmPlan{true, best_form, best_n, 0};
+  if (best_n == 0) return GemmPlan{false, 0, 0, 0, false};
+  return GemmPlan{true, best_form, best_n, 0, halves};
 }
 
 namespace {
@@ -492,7 +530,7 @@ namespace {
 template <bool kPair, int kTileN>
 cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, int64_t n,
                         const CUtensorMap& map_a, const CUtensorMap& map_b,
-                        const CUtensorMap& map_c, float* C, cudaStream_t stream) {
+                        const CUtensorMap& map_c, float* C, bool halves, cudaStream_t stream) {
   using S = Shape<kPair, kTileN>;
   const cudaError_t attr_err = set_smem_attribute<kPair, kTileN>();
   if (attr_err != cudaSuccess) return attr_err;
@@ -504,12 +542,22 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   p.m_tiles = (int)((m + S::kTileM - 1) / S::kTileM);
   p.n_tiles = (int)((n + kTileN - 1) / kTileN);
   p.tiles = b * p.m_tiles * (int64_t)p.n_tiles;
+  p.whole = p.tiles;
+  p.items = p.tiles;
   p.k_blocks = (int)((k + kTileK - 1) / kTileK);
   p.status = dev.status;
   p.a_box_rows = a_box_rows(m);
 
   const int64_t max_units = kPair ? pair_units(dev.sms) : dev.sms;
-  const int64_t units = std::min<int64_t>(p.tiles, max_units);
+  // The last wave of a compute-bound problem: when its tiles would occupy at most half the
+  // units, each is cut into two column halves so that twice as many units share the wave.
+  // (k is never cut: a second addition into C would make the bits depend on arrival order.)
+  const int64_t tail = p.tiles % max_units;
+  if (halves && (S::kColsB / 2) % 64 == 0 && p.tiles > max_units && tail > 0 && 2 * tail <= max_units) {
+    p.whole = p.tiles - tail;
+    p.items = p.whole + 2 * tail;
+  }
+  const int64_t units = std::min<int64_t>(p.items, max_units);
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(units * S::kCtas), 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
@@ -541,11 +589,11 @@ cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, 
   if (e != cudaSuccess) return e;
   const int code = plan.form * 1000 + plan.tile_n;
   switch (code) {
-    case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, C, stream); break;
-    case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, stream); break;
-    case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, stream); break;
-    case 2128: e = launch_gemm<true, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, stream); break;
-    case 2256: e = launch_gemm<true, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, stream); break;
+    case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, stream); break;
+    case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, stream); break;
+    case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, stream); break;
+    case 2128: e = launch_gemm<true, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, stream); break;
+    case 2256: e = launch_gemm<true, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, stream); break;
     default: return cudaErrorInvalidValue;
   }
   if (e == cudaSuccess) ++*launches;

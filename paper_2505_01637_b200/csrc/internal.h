@@ -73,11 +73,13 @@ struct GemmPlan {
   int form;      // 1: one CTA per 128-row tile, 2: a CTA pair per 256-row tile
   int tile_n;    // 64, 128 or 256 columns per tile
   size_t workspace_bytes;
+  bool halves;   // tiles of a sparse last wave may be cut into column halves
 };
 
 bool gemm_shape_supported(int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
                           const void* B, const void* C);
-// `knob`: 0 = by shape; otherwise form + 16 * (tile columns / 64), either part 0 = by shape.
+// `knob`: 0 = by shape; otherwise form + 16 * (tile columns / 64) [+ 256 to keep the last wave's
+// tiles whole], the first two parts 0 = by shape.
 GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob);
 // CTA pairs (cta_group::2) the current device can hold at once.
 int gemm_pair_units(int sms);

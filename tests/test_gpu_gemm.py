@@ -35,6 +35,22 @@ def test_integer_inputs_bit_exact(shape, form):
     check_full(A, B, C, integer=True, path=TC, split_k=form, what="tcgen05 form %d %s" % (form, shape))
 
 
+@pytest.mark.parametrize("shape,form", [
+    ((2, 1100, 72, 4504), 64 + 2),    # 180 pair tiles on 74 pairs: the last 32 are cut into halves; ragged n
+    ((1, 1280, 72, 4504), 64 + 1),    # 180 one-CTA tiles on 148 SMs: same, halves of 128 columns
+    ((1, 4096, 128, 4096), 0),        # the square config's tiling (256 tiles, 34 in the last wave), by shape
+    ((1, 2432, 64, 2048), 32 + 1),    # 128-column tiles cut into 64-column halves
+])
+def test_last_wave_cut_into_column_halves(shape, form):
+    b, m, k, n = shape
+    A, B, C = w.make(b, m, k, n, seed=sum(shape), ab="int4", c="normal")
+    cut = check_full(A, B, C, integer=True, path=TC, split_k=form, what="halves %s" % (shape,))
+    whole = gpu_run(A, B, C, path=TC, split_k=form + 256)
+    assert_bit_exact(whole, cut, "whole tiles vs halves %s" % (shape,))
+    A, B, C = w.make(b, m, k, n, seed=sum(shape) + 1, ab="normal_rsqrtk", c="normal0.1")
+    check_full(A, B, C, integer=False, path=TC, split_k=form, what="halves %s random" % (shape,))
+
+
 @pytest.mark.parametrize("form", [1, 2])
 def test_one_hot_operands_pin_the_operand_layouts(form):
     b, m, k, n = 2, 160, 136, 328
