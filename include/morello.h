@@ -135,8 +135,8 @@ size_t morello_noalloc_scratch_limit(void);
 /* --- introspection and experiments (tests and benchmarks) ------------------ */
 
 /* The path the selector picks for this shape with 16-byte-aligned operands:
- * MORELLO_PATH_SKINNY or MORELLO_PATH_TCGEN05 (-1 for an invalid shape).  One and two
- * rows go to the FP32-FMA kernels; from 3 rows on the tcgen05 kernel runs whenever it can
+ * MORELLO_PATH_SKINNY or MORELLO_PATH_TCGEN05 (-1 for an invalid shape).  A single row
+ * (the GEMV) goes to the FP32-FMA kernels; from 2 rows on the tcgen05 kernels run whenever they can
  * address the shape (k % 8 == 0, n % 8 == 0) and, up to 16 rows, B has enough columns
  * to give half the SMs a tile (the choice uses the current device's SM count, 148 when
  * no device is usable). */
@@ -151,7 +151,8 @@ int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n);
  * stages within 32 KiB: 16384 / m rows of k per block, m rounded up to 1, 2 or 4).  On the tcgen05 path, which never
  * splits k, the argument instead selects the tile: (value % 16) is the form -- 0 = by
  * shape, 1 = one CTA per 128-row tile, 2 = a pair of CTAs per 256-row tile
- * (cta_group::2) -- ((value / 16) % 16) is the tile's column count / 64 -- 0 = by
+ * (cta_group::2), 3 = the operand-swapped kernel for at most 64 rows (no column count
+ * with it) -- ((value / 16) % 16) is the tile's column count / 64 -- 0 = by
  * shape, 1, 2 or 4 (64 columns only with form 1) -- and adding 256 keeps the tiles of a
  * sparse last wave whole instead of cutting them into column halves.  Returns MORELLO_ERR_UNSUPPORTED_PATH, and
  * enqueues nothing, when the path cannot run the shape (the tcgen05 path needs

@@ -89,13 +89,13 @@ int validate(int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const vo
 }
 
 // Measured on the 2048 x 16384 weight shape (us per call, FMA kernels / tensor path):
-// m = 1: 11.0 / 13.9, m = 2: 11.6 / 14.0, m = 4: 16.6 / 14.1, m = 8: 35.6 / 14.1,
-// m = 16: 84.8 / 14.2.  Every extra row costs the FMA kernels one FMA per element of B
-// while the tensor cores take up to 128 rows for the price of one, so the FMA kernels keep
-// one and two rows only.  Between 3 and 16 rows the tensor path still needs enough column
-// tiles to occupy the device; a tall and narrow B (few columns, long k) is better served by
-// the FMA kernel's split of k.
-constexpr int kFmaMaxRows = 2;
+// m = 1: 10.98 / 11.26, m = 2: 11.79 / 11.38, m = 4: 16.6 / 11.4, m = 8: 35.6 / 11.5,
+// m = 16: 84.8 / 11.7.  Every extra row costs the FMA kernels one FMA per element of B
+// while the tensor cores take the rows for free, so the FMA kernels keep the single row (the
+// GEMV proper).  Up to 16 rows the tensor path still needs enough column tiles to occupy the
+// device; a tall and narrow B (few columns, long k) is better served by the FMA kernel's
+// split of k.
+constexpr int kFmaMaxRows = 1;
 int select_path(int sms, int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const void* B,
                 const void* C) {
   if (m <= kFmaMaxRows) return MORELLO_PATH_SKINNY;

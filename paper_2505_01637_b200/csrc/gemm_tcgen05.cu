@@ -352,6 +352,184 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// Few rows (m <= 64): the operands trade places.  C^T[n, m] += B^T[n, k] x A^T[k, m]: a thread
+// block owns a strip of 128 columns of B, which becomes the M side of the MMA (B is [k][n], so
+// it is the MN-major operand here too: two TMA boxes of 64 k rows x 64 columns per k block,
+// the same boxes the tiles above use), and the rows of A, rounded up to a multiple of 16,
+// are its N side (K-major, one box of 64 k x kRowsA rows per k block).  The MMA's cost then
+// follows m instead of a fixed 128 rows, the accumulator is 128 lanes x kRowsA columns, and
+// the epilogue holds one column of C per thread: for every row i a warp adds 32 consecutive
+// floats of C (C is read before the main loop, the sum is added once, at the end).
+// The call streams B once and is bound by HBM, so the block is kept small enough (at most
+// 108 KiB of stages, 32 or 64 TMEM columns) for the next call's block to be resident beside
+// it: before its griddepcontrol.wait that block asks the TMA engine to prefetch its first k
+// blocks of B into L2 (nothing reaches the SM, so this is legal early), and a block lets
+// dependents launch once its producer has issued its last load.
+#ifndef MORELLO_SWAP_RING_KIB
+#define MORELLO_SWAP_RING_KIB 108        // shared memory for the stages: two blocks fit an SM
+#endif
+#ifndef MORELLO_SWAP_PREFETCH_BLOCKS
+#define MORELLO_SWAP_PREFETCH_BLOCKS 6
+#endif
+template <int kRowsA>
+struct SwapShape {
+  static constexpr int kBytesStrip = 2 * kBoxBytesB;                  // 128 columns x 64 k: 16 KiB
+  static constexpr int kBytesRows = kRowsA * kTileK * 2;              // 2 .. 8 KiB
+  static constexpr int kStageBytes = kBytesStrip + kBytesRows;
+  static constexpr int kFit = (MORELLO_SWAP_RING_KIB * 1024) / kStageBytes;
+  static constexpr int kStages = kFit < kMaxStages ? kFit : kMaxStages;
+  static constexpr int kTmemCols = kRowsA <= 32 ? 32 : 64;
+  static constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256;
+  static_assert(kRowsA % 16 == 0 && kRowsA >= 16 && kRowsA <= 64, "rows of A");
+};
+constexpr int kSwapStripCols = 128;
+constexpr int kSwapAutoRows = 32;        // the planner picks this kernel up to this many rows
+constexpr int kSwapPrefetchBlocks = MORELLO_SWAP_PREFETCH_BLOCKS;   // k blocks asked into L2 before the wait
+
+struct SwapParams {
+  float* C;
+  int64_t m, n;
+  int64_t c_batch;  // m * n
+  int k_blocks;
+  uint32_t* status;
+};
+
+struct SwapBarriers {
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
+  uint64_t acc_full;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+template <int kRowsA>
+__global__ void __launch_bounds__(kThreads)
+swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+            const SwapParams p) {
+  using S = SwapShape<kRowsA>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* stages = reinterpret_cast<uint8_t*>(
+      (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  SwapBarriers* bars = reinterpret_cast<SwapBarriers*>(stages + (size_t)S::kStages * S::kStageBytes);
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int col0 = blockIdx.x * kSwapStripCols;
+  const int bb = blockIdx.y;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S::kStages; ++s) {
+      mbar_init(&bars->full[s], 1);
+      mbar_init(&bars->empty[s], 1);
+    }
+    mbar_init(&bars->acc_full, 1);
+    bars->abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_descriptor(&map_a);
+    tma_prefetch_descriptor(&map_b);
+    const int ahead = min(p.k_blocks, kSwapPrefetchBlocks);
+    for (int kb = 0; kb < ahead; ++kb) {
+      tma_prefetch_l2_3d(&map_b, col0, kb * kTileK, bb);
+      tma_prefetch_l2_3d(&map_b, col0 + 64, kb * kTileK, bb);
+    }
+  }
+  if (warp == 1) {
+    tmem_alloc(&bars->tmem_base, S::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  // Nothing above read or wrote global memory; from here on the predecessor on the stream has
+  // completed.
+  pdl_wait();
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (elect_one()) {
+      int stage = 0;
+      uint32_t phase = 0;
+      for (int kb = 0; kb < p.k_blocks; ++kb) {
+        if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag, p.status, 8)) break;
+        uint8_t* sb = stages + (size_t)stage * S::kStageBytes;
+        uint8_t* sa = sb + S::kBytesStrip;
+        mbar_arrive_expect_tx(&bars->full[stage], S::kStageBytes);
+        tma_load_3d(sb, &map_b, &bars->full[stage], col0, kb * kTileK, bb);
+        tma_load_3d(sb + kBoxBytesB, &map_b, &bars->full[stage], col0 + 64, kb * kTileK, bb);
+        tma_load_3d(sa, &map_a, &bars->full[stage], kb * kTileK, 0, bb);
+        if (++stage == S::kStages) { stage = 0; phase ^= 1; }
+      }
+      // Every load of this block is in flight: the next kernel's blocks may come in.
+      pdl_release();
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (elect_one()) {
+      // M = 128 columns of B (MN-major A operand), N = kRowsA rows of A (K-major B operand).
+      constexpr uint32_t idesc = instr_desc_bf16(kSwapStripCols, kRowsA, true, false);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int kb = 0; kb < p.k_blocks; ++kb) {
+        if (!(ok = mbar_wait(&bars->full[stage], phase, abort_flag, p.status, 9))) break;
+        tc_fence_after_sync();
+        const uint32_t sb = smem_u32(stages + (size_t)stage * S::kStageBytes);
+        const uint32_t sa = sb + S::kBytesStrip;
+#pragma unroll
+        for (int j = 0; j < kTileK / 16; ++j) {
+          // The strip of B: 64-column groups one TMA box apart, 8-row k groups 1024 bytes
+          // apart, 16 k rows = 2048 bytes.  The rows of A: 8-row groups 1024 bytes apart,
+          // 16 k elements = 32 bytes along the row.
+          const uint64_t d_strip = smem_desc_sw128(sb + j * 2048, kBoxBytesB, 1024);
+          const uint64_t d_rows = smem_desc_sw128(sa + j * 32, 16, 1024);
+          mma_bf16_ss(tmem_base, d_strip, d_rows, idesc, (kb | j) != 0 ? 1u : 0u);
+        }
+        mma_commit(&bars->empty[stage]);
+        if (++stage == S::kStages) { stage = 0; phase ^= 1; }
+      }
+      if (ok) mma_commit(&bars->acc_full);
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int quarter = warp & 3;  // TMEM lanes [32 * quarter, 32 * quarter + 32)
+    const int64_t col = (int64_t)col0 + quarter * 32 + lane;   // this thread's column of C
+    const bool col_live = col < p.n;
+    float* c_col = p.C + (int64_t)bb * p.c_batch + col;
+    float c_in[kRowsA];
+#pragma unroll
+    for (int i = 0; i < kRowsA; ++i) c_in[i] = (col_live && i < p.m) ? c_col[(int64_t)i * p.n] : 0.f;
+    bool ok = mbar_wait(&bars->acc_full, 0, abort_flag, p.status, 10);
+    ok = __all_sync(0xffffffffu, ok);  // also reconverges the warp for the aligned TMEM loads
+    if (ok) {
+      tc_fence_after_sync();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll
+      for (int g = 0; g < kRowsA / 16; ++g) {
+        uint32_t r[16];
+        tmem_ld_32x16(taddr + g * 16, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          if (col_live && g * 16 + i < p.m)
+            c_col[(int64_t)(g * 16 + i) * p.n] = c_in[g * 16 + i] + __uint_as_float(r[i]);
+      }
+    }
+  }
+
+  __syncwarp();
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc(tmem_base, S::kTmemCols);
+  }
+}
+
 // Tensor maps are cached per (pointers, shape): encoding one costs a few microseconds.
 struct MapKey {
   const void* a;
@@ -491,6 +669,15 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t, int64_t n, int knob) 
   const bool halves = (knob / 256) == 0;
   knob %= 256;
   int form = knob % 16, tile_n = (knob / 16) * 64;
+  // Form 3: the operand-swapped kernel for few rows.  By shape it takes every call of at most
+  // 32 rows whose strips of 128 columns occupy at least half the SMs (measured on 2048 x 16384,
+  // us per call, swapped / 128-row tiles: m = 16: 11.7 / 14.2, 32: 12.7 / 14.4, 48: 14.6 / 14.6,
+  // 64: 15.5 / 14.8 -- with more rows of A per stage the ring gets shallower).
+  if (form == 3 || (form == 0 && tile_n == 0 && m <= kSwapAutoRows && b <= 65535 &&
+                    b * ((n + kSwapStripCols - 1) / kSwapStripCols) * 2 >= sms)) {
+    if (m > 64 || tile_n != 0 || b > 65535) return GemmPlan{false, 0, 0, 0, false};
+    return GemmPlan{true, 3, a_box_rows(m), 0, false};
+  }
   if (form < 0 || form > 2 || (tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) ||
       (form == 2 && tile_n == 64))
     return GemmPlan{false, 0, 0, 0, false};
@@ -581,6 +768,49 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
 
 }  // namespace
 
+namespace {
+
+template <int kRowsA>
+cudaError_t launch_swap(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, int64_t n,
+                        const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
+                        cudaStream_t stream, uint64_t* launches) {
+  using S = SwapShape<kRowsA>;
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [] {
+    attr_err = cudaFuncSetAttribute(swap_kernel<kRowsA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)S::kSmemBytes);
+  });
+  if (attr_err != cudaSuccess) return attr_err;
+  SwapParams p{};
+  p.m = m; p.n = n;
+  p.c_batch = m * n;
+  p.k_blocks = (int)((k + kTileK - 1) / kTileK);
+  p.status = dev.status;
+  const int64_t strips = (n + kSwapStripCols - 1) / kSwapStripCols;
+  // grid.y carries the batch index (the tensor maps cover all batches); larger batches in slabs
+  for (int64_t b0 = 0; b0 < b; b0 += 65535) {
+    if (b0 != 0) return cudaErrorInvalidValue;   // the planner keeps such batches off this form
+    p.C = C;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)strips, (unsigned)std::min<int64_t>(b, 65535), 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = S::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, swap_kernel<kRowsA>, map_a, map_b, p);
+    if (e != cudaSuccess) return e;
+    ++*launches;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace
+
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m, int64_t k,
                         int64_t n, const uint16_t* A, const uint16_t* B, float* C, float*,
                         cudaStream_t stream, uint64_t* launches) {
@@ -589,6 +819,10 @@ cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, 
   if (e != cudaSuccess) return e;
   const int code = plan.form * 1000 + plan.tile_n;
   switch (code) {
+    case 3016: return launch_swap<16>(dev, b, m, k, n, map_a, map_b, C, stream, launches);
+    case 3032: return launch_swap<32>(dev, b, m, k, n, map_a, map_b, C, stream, launches);
+    case 3048: return launch_swap<48>(dev, b, m, k, n, map_a, map_b, C, stream, launches);
+    case 3064: return launch_swap<64>(dev, b, m, k, n, map_a, map_b, C, stream, launches);
     case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, stream); break;
     case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, stream); break;
     case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, stream); break;

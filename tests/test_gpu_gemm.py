@@ -120,3 +120,65 @@ def test_repeated_calls_give_identical_bits_and_accumulate(form):
     A, B, C = w.make(b, m, k, n, seed=6, ab="int4", c="int8")
     twice = oracle.matmul_accum(b, m, k, n, A, B, oracle.matmul_accum(b, m, k, n, A, B, C))
     assert_bit_exact(gpu_run(A, B, C, path=TC, split_k=form, calls=2), twice, "two accumulating calls")
+
+
+# ------------------------------------------------ the operand-swapped kernel for few rows (form 3)
+SWAP = 3
+
+
+@pytest.mark.parametrize("shape", [
+    (1, 1, 64, 128),        # one strip, one k block, one row
+    (1, 16, 16, 128),       # one MMA instruction's worth of k
+    (1, 3, 640, 256),       # the stage ring wraps
+    (2, 16, 200, 264),      # ragged k and n, batches
+    (3, 17, 72, 136),       # 17 rows: the 32-row instantiation
+    (1, 33, 264, 520),      # 48-row instantiation
+    (1, 49, 128, 392),      # 64-row instantiation
+    (1, 64, 2048, 1024),
+    (1, 16, 2048, 16384),   # the decode-style config
+])
+def test_swap_form_matches_oracle(shape):
+    b, m, k, n = shape
+    A, B, C = w.make(b, m, k, n, seed=sum(shape), ab="int4", c="normal")
+    check_full(A, B, C, integer=True, path=TC, split_k=SWAP, what="swap form %s" % (shape,))
+    A, B, C = w.make(b, m, k, n, seed=sum(shape) + 1, ab="uniform_rsqrtk", c="normal")
+    check_full(A, B, C, integer=False, path=TC, split_k=SWAP, what="swap form %s random" % (shape,))
+
+
+def test_swap_form_one_hot_operands_and_repeatability():
+    b, m, k, n = 2, 20, 136, 328
+    rng = np.random.default_rng(7)
+    Bv = rng.integers(-100, 101, size=(b, k, n)).astype(np.float32)
+    Av = rng.integers(-100, 101, size=(b, m, k)).astype(np.float32)
+    C = rng.integers(-50, 51, size=(b, m, n)).astype(np.float32)
+    for (b0, i0, p0) in [(0, 0, 0), (0, 19, 70), (1, 7, 135), (1, 16, 64)]:
+        A1 = np.zeros((b, m, k), np.float32)
+        A1[b0, i0, p0] = 2.0
+        want = C.copy()
+        want[b0, i0, :] += 2.0 * Bv[b0, p0, :]
+        got = gpu_run(w.f32_to_bf16_rne(A1), w.f32_to_bf16_rne(Bv), C, path=TC, split_k=SWAP)
+        assert_bit_exact(got, want, "swap one-hot A at %s" % ((b0, i0, p0),))
+    for (b0, p0, j0) in [(0, 0, 0), (0, 70, 201), (1, 135, 327), (1, 64, 128)]:
+        B1 = np.zeros((b, k, n), np.float32)
+        B1[b0, p0, j0] = -3.0
+        want = C.copy()
+        want[b0, :, j0] += -3.0 * Av[b0, :, p0]
+        got = gpu_run(w.f32_to_bf16_rne(Av), w.f32_to_bf16_rne(B1), C, path=TC, split_k=SWAP)
+        assert_bit_exact(got, want, "swap one-hot B at %s" % ((b0, p0, j0),))
+    A, B, C = w.make(1, 16, 1024, 2048, seed=8, ab="normal_rsqrtk", c="normal")
+    first = gpu_run(A, B, C, path=TC, split_k=SWAP)
+    for _ in range(3):
+        assert np.array_equal(bits(gpu_run(A, B, C, path=TC, split_k=SWAP)), bits(first))
+    A, B, C = w.make(1, 16, 1024, 2048, seed=9, ab="int4", c="int8")
+    twice = oracle.matmul_accum(1, 16, 1024, 2048, A, B, oracle.matmul_accum(1, 16, 1024, 2048, A, B, C))
+    assert_bit_exact(gpu_run(A, B, C, path=TC, split_k=SWAP, calls=2), twice, "swap form, two accumulating calls")
+
+
+def test_swap_form_refuses_more_than_64_rows():
+    b, m, k, n = 1, 65, 64, 128
+    A, B, C = w.make(b, m, k, n, seed=1)
+    from gpu_util import to_dev
+    dA, dB, dC = to_dev(A, B, C)
+    with pytest.raises(mb.MorelloError) as e:
+        mb.morello_matmul_accum_forced(TC, SWAP, b, m, k, n, dA, dB, dC)
+    assert e.value.status == mb.MORELLO_ERR_UNSUPPORTED_PATH
