@@ -90,6 +90,26 @@ int morello_matmul_accum_ws(int64_t b, int64_t m, int64_t k, int64_t n,
                             void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Matmul(b x m x k x n), the non-accumulating member of the pair (Section 2.2 of the
+ * paper lists Matmul beside MatmulAccum; Matmul is MatmulAccum into a zeroed output):
+ *
+ *     C[b,i,j]  <-  sum_{p<k} A[b,i,p] * B[b,p,j]
+ *
+ * Same layouts, kernels, scratch rules and status codes as morello_matmul_accum.  C is
+ * write-only: its prior contents are neither read nor added (the kernels skip the read,
+ * which on large outputs is a third of the memory traffic).  k == 0 sets C to zero;
+ * b*m*n == 0 does nothing.
+ */
+int morello_matmul(int64_t b, int64_t m, int64_t k, int64_t n,
+                   const void* A, const void* B, float* C, void* stream);
+
+/* morello_matmul on a given path / split / tile: arguments as morello_matmul_accum_forced. */
+int morello_matmul_forced(int path, int split_k,
+                          int64_t b, int64_t m, int64_t k, int64_t n,
+                          const void* A, const void* B, float* C,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * End-to-end convenience call on HOST buffers (same layouts): copies A, B and
  * C to library-owned device staging (grown on demand), runs the operation,
  * copies C back and synchronises before returning.  Pinned host memory makes

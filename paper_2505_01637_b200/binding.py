@@ -34,6 +34,9 @@ _i64, _vp, _int, _sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_s
 # name -> (restype, argtypes); mirrors include/morello.h declaration by declaration
 SIGNATURES = {
     "morello_matmul_accum": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
+    "morello_matmul": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
+    "morello_matmul_forced": (_int, [_int, _int, _i64, _i64, _i64, _i64, _vp, _vp, _vp,
+                                     _vp, _sz, _vp]),
     "morello_workspace_bytes": (_sz, [_i64, _i64, _i64, _i64]),
     "morello_matmul_accum_ws": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _sz, _vp]),
     "morello_matmul_accum_host": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp]),
@@ -112,6 +115,19 @@ def _check(status: int, where: str) -> None:
 def morello_matmul_accum(b, m, k, n, A, B, C, stream=None) -> None:
     _check(lib().morello_matmul_accum(b, m, k, n, _addr(A), _addr(B), _addr(C), _stream(stream)),
            "morello_matmul_accum")
+
+
+def morello_matmul(b, m, k, n, A, B, C, stream=None) -> None:
+    """C = A x B (C's prior contents are not read)."""
+    _check(lib().morello_matmul(b, m, k, n, _addr(A), _addr(B), _addr(C), _stream(stream)),
+           "morello_matmul")
+
+
+def morello_matmul_forced(path, split_k, b, m, k, n, A, B, C, workspace=None,
+                          workspace_bytes=0, stream=None) -> None:
+    _check(lib().morello_matmul_forced(path, split_k, b, m, k, n, _addr(A), _addr(B), _addr(C),
+                                       _addr(workspace), workspace_bytes, _stream(stream)),
+           "morello_matmul_forced")
 
 
 def morello_workspace_bytes(b, m, k, n) -> int:

@@ -148,7 +148,7 @@ size_t workspace_for(int sms, int path, int knob, int64_t b, int64_t m, int64_t 
 
 int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
         const void* B, float* C, void* workspace, size_t workspace_bytes, bool own_scratch,
-        void* stream) {
+        void* stream, bool overwrite = false) {
   bool empty = false;
   int rc = validate(b, m, k, n, A, B, C, &empty);
   if (rc != MORELLO_OK) return rc;
@@ -161,7 +161,16 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     rc = device_state(&st);
   }
   if (rc != MORELLO_OK) return rc;
-  if (empty) return MORELLO_OK;
+  if (empty) {
+    // An empty sum: MatmulAccum leaves C alone, Matmul sets it to zero.
+    if (overwrite && b > 0 && m > 0 && n > 0) {
+      if (!C) return MORELLO_ERR_NULL_POINTER;
+      if (reinterpret_cast<uintptr_t>(C) % 4) return MORELLO_ERR_MISALIGNED;
+      const cudaError_t e = cudaMemsetAsync(C, 0, (size_t)b * m * n * 4, static_cast<cudaStream_t>(stream));
+      if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return MORELLO_OK;
+  }
 
   if (path == MORELLO_PATH_AUTO) {
     path = select_path(st->info.sms, b, m, k, n, A, B, C);
@@ -210,11 +219,11 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     const GemmPlan plan = gemm_plan(sms, b, m, k, n, split_k);
     if (!plan.supported) return MORELLO_ERR_UNSUPPORTED_PATH;
     e = gemm_launch(st->info, plan, b, m, k, n, static_cast<const uint16_t*>(A),
-                    static_cast<const uint16_t*>(B), C, ws, s, &launches);
+                    static_cast<const uint16_t*>(B), C, ws, s, &launches, overwrite);
   } else if (which == SKINNY_STREAM) {
     const StreamPlan plan = stream_plan(sms, b, (int)m, k, n, split_k % kKnobSplitMod);
     e = stream_launch(st->info, plan, b, (int)m, k, n, static_cast<const uint16_t*>(A), m * k,
-                      static_cast<const uint16_t*>(B), C, m * n, ws, s, &launches);
+                      static_cast<const uint16_t*>(B), C, m * n, ws, s, &launches, overwrite);
   } else {
     const uint16_t* a = static_cast<const uint16_t*>(A);
     const int split = split_k % kKnobSplitMod;
@@ -222,7 +231,7 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
       const int mc = (int)std::min<int64_t>(kSkinnyMaxRows, m - i0);
       const SkinnyPlan plan = skinny_plan(sms, b, mc, k, n, vec, split);
       e = skinny_launch(plan, b, mc, k, n, a + i0 * k, m * k, static_cast<const uint16_t*>(B),
-                        C + i0 * n, m * n, ws, s, &launches);
+                        C + i0 * n, m * n, ws, s, &launches, overwrite);
     }
   }
   g_launches.fetch_add(launches, std::memory_order_relaxed);
@@ -275,6 +284,18 @@ int morello_matmul_accum_forced(int path, int split_k, int64_t b, int64_t m, int
                                 size_t workspace_bytes, void* stream) {
   const bool own = (workspace == nullptr && workspace_bytes == 0);
   return run(path, split_k, b, m, k, n, A, B, C, workspace, workspace_bytes, own, stream);
+}
+
+int morello_matmul(int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const void* B,
+                   float* C, void* stream) {
+  return run(MORELLO_PATH_AUTO, 0, b, m, k, n, A, B, C, nullptr, 0, true, stream, true);
+}
+
+int morello_matmul_forced(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n,
+                          const void* A, const void* B, float* C, void* workspace,
+                          size_t workspace_bytes, void* stream) {
+  const bool own = (workspace == nullptr && workspace_bytes == 0);
+  return run(path, split_k, b, m, k, n, A, B, C, workspace, workspace_bytes, own, stream, true);
 }
 
 int morello_matmul_accum_host(int64_t b, int64_t m, int64_t k, int64_t n, const void* A_host,

@@ -80,6 +80,7 @@ struct GemmParams {
   int64_t items;    // items [whole, items) are the column halves of tiles [whole, tiles)
   int k_blocks;
   uint32_t* status;
+  int overwrite;   // 1: C = product (TMA store) instead of C += product (TMA reduce-add)
   int a_box_rows;  // rows of A one TMA box brings: 128, or m rounded up to 16 when m < 128
 };
 
@@ -324,7 +325,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           if (lane == 0) {
             // C[bb, row0 : row0 + 32, col0 + c : col0 + c + 32] += block; rows and columns
             // past the edge of C are dropped by the TMA engine.
-            tma_reduce_add_3d(&map_c, my_blocks + blk * kEpiBlockBytes, col0 + c, row0, bb);
+            if (p.overwrite) tma_store_3d(&map_c, my_blocks + blk * kEpiBlockBytes, col0 + c, row0, bb);
+            else tma_reduce_add_3d(&map_c, my_blocks + blk * kEpiBlockBytes, col0 + c, row0, bb);
             bulk_commit_group();
           }
           blk ^= 1u;
@@ -389,6 +391,7 @@ constexpr int kSwapPrefetchBlocks = MORELLO_SWAP_PREFETCH_BLOCKS;   // k blocks 
 
 struct SwapParams {
   float* C;
+  int overwrite;    // 1: C = product instead of C += product
   int64_t m, n;
   int64_t c_batch;  // m * n
   int k_blocks;
@@ -501,7 +504,8 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     float* c_col = p.C + (int64_t)bb * p.c_batch + col;
     float c_in[kRowsA];
 #pragma unroll
-    for (int i = 0; i < kRowsA; ++i) c_in[i] = (col_live && i < p.m) ? c_col[(int64_t)i * p.n] : 0.f;
+    for (int i = 0; i < kRowsA; ++i)
+      c_in[i] = (col_live && i < p.m && !p.overwrite) ? c_col[(int64_t)i * p.n] : 0.f;
     bool ok = mbar_wait(&bars->acc_full, 0, abort_flag, p.status, 10);
     ok = __all_sync(0xffffffffu, ok);  // also reconverges the warp for the aligned TMEM loads
     if (ok) {
@@ -717,7 +721,8 @@ namespace {
 template <bool kPair, int kTileN>
 cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, int64_t n,
                         const CUtensorMap& map_a, const CUtensorMap& map_b,
-                        const CUtensorMap& map_c, float* C, bool halves, cudaStream_t stream) {
+                        const CUtensorMap& map_c, float* C, bool halves, bool overwrite,
+                        cudaStream_t stream) {
   using S = Shape<kPair, kTileN>;
   const cudaError_t attr_err = set_smem_attribute<kPair, kTileN>();
   if (attr_err != cudaSuccess) return attr_err;
@@ -734,6 +739,7 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   p.k_blocks = (int)((k + kTileK - 1) / kTileK);
   p.status = dev.status;
   p.a_box_rows = a_box_rows(m);
+  p.overwrite = overwrite ? 1 : 0;
 
   const int64_t max_units = kPair ? pair_units(dev.sms) : dev.sms;
   // The last wave of a compute-bound problem: when its tiles would occupy at most half the
@@ -773,7 +779,7 @@ namespace {
 template <int kRowsA>
 cudaError_t launch_swap(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, int64_t n,
                         const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
-                        cudaStream_t stream, uint64_t* launches) {
+                        bool overwrite, cudaStream_t stream, uint64_t* launches) {
   using S = SwapShape<kRowsA>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
@@ -783,6 +789,7 @@ cudaError_t launch_swap(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   });
   if (attr_err != cudaSuccess) return attr_err;
   SwapParams p{};
+  p.overwrite = overwrite ? 1 : 0;
   p.m = m; p.n = n;
   p.c_batch = m * n;
   p.k_blocks = (int)((k + kTileK - 1) / kTileK);
@@ -813,21 +820,21 @@ cudaError_t launch_swap(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
 
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m, int64_t k,
                         int64_t n, const uint16_t* A, const uint16_t* B, float* C, float*,
-                        cudaStream_t stream, uint64_t* launches) {
+                        cudaStream_t stream, uint64_t* launches, bool overwrite) {
   CUtensorMap map_a, map_b, map_c;
   cudaError_t e = get_maps(MapKey{A, B, C, b, m, k, n}, &map_a, &map_b, &map_c);
   if (e != cudaSuccess) return e;
   const int code = plan.form * 1000 + plan.tile_n;
   switch (code) {
-    case 3016: return launch_swap<16>(dev, b, m, k, n, map_a, map_b, C, stream, launches);
-    case 3032: return launch_swap<32>(dev, b, m, k, n, map_a, map_b, C, stream, launches);
-    case 3048: return launch_swap<48>(dev, b, m, k, n, map_a, map_b, C, stream, launches);
-    case 3064: return launch_swap<64>(dev, b, m, k, n, map_a, map_b, C, stream, launches);
-    case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, stream); break;
-    case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, stream); break;
-    case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, stream); break;
-    case 2128: e = launch_gemm<true, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, stream); break;
-    case 2256: e = launch_gemm<true, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, stream); break;
+    case 3016: return launch_swap<16>(dev, b, m, k, n, map_a, map_b, C, overwrite, stream, launches);
+    case 3032: return launch_swap<32>(dev, b, m, k, n, map_a, map_b, C, overwrite, stream, launches);
+    case 3048: return launch_swap<48>(dev, b, m, k, n, map_a, map_b, C, overwrite, stream, launches);
+    case 3064: return launch_swap<64>(dev, b, m, k, n, map_a, map_b, C, overwrite, stream, launches);
+    case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, stream); break;
+    case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, stream); break;
+    case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, stream); break;
+    case 2128: e = launch_gemm<true, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, stream); break;
+    case 2256: e = launch_gemm<true, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, stream); break;
     default: return cudaErrorInvalidValue;
   }
   if (e == cudaSuccess) ++*launches;

@@ -78,6 +78,7 @@ struct StreamParams {
   int strips;
   int split_k;
   int k_per_split;                // multiple of kBoxRows
+  int overwrite;                  // 1: C = sum instead of C += sum
   int a_bulk;                     // rows of A can be brought by bulk copies (16-byte alignment)
   uint32_t* status;
 };
@@ -194,7 +195,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_b, const StreamParams
     const int i = o / kStripCols;
     const int64_t col = col0 + (o % kStripCols);
     c_in[r] = 0.f;
-    if (p.split_k == 1 && o < M_T * kStripCols && i < p.m && col < p.n)
+    if (p.split_k == 1 && !p.overwrite && o < M_T * kStripCols && i < p.m && col < p.n)
       c_in[r] = p.C[(int64_t)bb * p.c_batch + (int64_t)i * p.n + col];
   }
   consumer_sync();
@@ -399,8 +400,9 @@ StreamPlan stream_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int spli
 cudaError_t stream_launch(const DeviceInfo& dev, const StreamPlan& plan, int64_t b, int m, int64_t k,
                           int64_t n, const uint16_t* A, int64_t a_batch, const uint16_t* B, float* C,
                           int64_t c_batch, float* workspace, cudaStream_t stream,
-                          uint64_t* launches) {
+                          uint64_t* launches, bool overwrite) {
   StreamParams prm{};
+  prm.overwrite = overwrite ? 1 : 0;
   prm.a_batch = a_batch; prm.c_batch = c_batch;
   prm.k = k; prm.n = n;
   prm.partial_split_stride = b * m * n;
@@ -428,7 +430,7 @@ cudaError_t stream_launch(const DeviceInfo& dev, const StreamPlan& plan, int64_t
     ++*launches;
   }
   if (plan.split_k > 1) {
-    cudaError_t e = skinny_reduce_launch(workspace, C, b, m, n, c_batch, plan.split_k, stream);
+    cudaError_t e = skinny_reduce_launch(workspace, C, b, m, n, c_batch, plan.split_k, stream, overwrite);
     if (e != cudaSuccess) return e;
     ++*launches;
   }

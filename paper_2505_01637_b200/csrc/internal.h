@@ -1,4 +1,6 @@
 // Internal declarations shared by the translation units of the CUDA library.
+// `overwrite` selects the non-accumulating operation everywhere: C = A x B, C's prior contents
+// neither read nor added.
 // Nothing here is visible through the C ABI.
 #pragma once
 
@@ -42,12 +44,13 @@ int skinny_vec(int64_t n, const void* B);
 cudaError_t skinny_launch(const SkinnyPlan& plan, int64_t b, int m, int64_t k, int64_t n,
                           const uint16_t* A, int64_t a_batch, const uint16_t* B, float* C,
                           int64_t c_batch, float* workspace, cudaStream_t stream,
-                          uint64_t* launches);
+                          uint64_t* launches, bool overwrite = false);
 
 // Enqueues the slice-ordered reduce: C[b, i, :] += partial[0] + partial[1] + ... for the
 // b * m * n sums of one row chunk (partial is [split_k][b][m][n], c_batch the batch stride of C).
 cudaError_t skinny_reduce_launch(const float* partial, float* C, int64_t b, int m, int64_t n,
-                                 int64_t c_batch, int split_k, cudaStream_t stream);
+                                 int64_t c_batch, int split_k, cudaStream_t stream,
+                                 bool overwrite = false);
 
 // ---- streaming GEMV (FP32 FMA, B through a TMA ring, m <= 4) ------------------
 struct StreamPlan {
@@ -65,7 +68,7 @@ StreamPlan stream_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int spli
 cudaError_t stream_launch(const DeviceInfo& dev, const StreamPlan& plan, int64_t b, int m, int64_t k,
                           int64_t n, const uint16_t* A, int64_t a_batch, const uint16_t* B, float* C,
                           int64_t c_batch, float* workspace, cudaStream_t stream,
-                          uint64_t* launches);
+                          uint64_t* launches, bool overwrite = false);
 
 // ---- tcgen05 path ------------------------------------------------------------
 struct GemmPlan {
@@ -85,6 +88,7 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob
 int gemm_pair_units(int sms);
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m,
                         int64_t k, int64_t n, const uint16_t* A, const uint16_t* B, float* C,
-                        float* workspace, cudaStream_t stream, uint64_t* launches);
+                        float* workspace, cudaStream_t stream, uint64_t* launches,
+                        bool overwrite = false);
 
 }  // namespace morello

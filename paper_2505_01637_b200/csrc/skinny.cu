@@ -40,6 +40,7 @@ struct SkinnyParams {
   int split_k;
   int k_chunk;
   int early_b;  // 1: B may be fetched before the preceding kernel on the stream has completed
+  int overwrite;  // 1: C = sum instead of C += sum
 };
 
 template <int M_T>
@@ -216,7 +217,7 @@ skinny_kernel(const SkinnyParams p) {
     for (int r = 1; r < R; ++r) sum += red[(size_t)r * W + o];
     if (p.split_k == 1) {
       float* c = p.C + (int64_t)bb * p.c_batch + (int64_t)i * p.n + col;
-      *c = *c + sum;
+      *c = p.overwrite ? sum : *c + sum;
     } else {
       p.partial[(int64_t)s * p.partial_split_stride + ((int64_t)bb * p.m + i) * p.n + col] = sum;
     }
@@ -226,7 +227,7 @@ skinny_kernel(const SkinnyParams p) {
 // C[b, i, :] += sum over slices, slice order fixed; one thread per output element.
 __global__ void __launch_bounds__(256)
 reduce_kernel(const float* __restrict__ partial, float* __restrict__ C, int64_t total,
-              int64_t mn, int64_t c_batch, int split_k) {
+              int64_t mn, int64_t c_batch, int split_k, int overwrite) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   pdl_wait();
   pdl_release();
@@ -235,7 +236,7 @@ reduce_kernel(const float* __restrict__ partial, float* __restrict__ C, int64_t 
   for (int s = 1; s < split_k; ++s) sum += partial[(int64_t)s * total + idx];
   const int64_t bb = idx / mn;
   float* c = C + bb * c_batch + (idx - bb * mn);
-  *c = *c + sum;
+  *c = overwrite ? sum : *c + sum;
 }
 
 // Launch with programmatic stream serialisation (see pdl_wait above).
@@ -346,8 +347,9 @@ SkinnyPlan skinny_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int vec,
 cudaError_t skinny_launch(const SkinnyPlan& plan, int64_t b, int m, int64_t k, int64_t n,
                           const uint16_t* A, int64_t a_batch, const uint16_t* B, float* C,
                           int64_t c_batch, float* workspace, cudaStream_t stream,
-                          uint64_t* launches) {
+                          uint64_t* launches, bool overwrite) {
   SkinnyParams prm{};
+  prm.overwrite = overwrite ? 1 : 0;
   prm.A = A; prm.B = B; prm.C = C; prm.partial = workspace;
   prm.a_batch = a_batch; prm.b_batch = k * n; prm.c_batch = c_batch;
   prm.k = k; prm.n = n;
@@ -378,7 +380,7 @@ cudaError_t skinny_launch(const SkinnyPlan& plan, int64_t b, int m, int64_t k, i
     ++*launches;
   }
   if (plan.split_k > 1) {
-    cudaError_t e = skinny_reduce_launch(workspace, C, b, m, n, c_batch, plan.split_k, stream);
+    cudaError_t e = skinny_reduce_launch(workspace, C, b, m, n, c_batch, plan.split_k, stream, overwrite);
     if (e != cudaSuccess) return e;
     ++*launches;
   }
@@ -386,11 +388,11 @@ cudaError_t skinny_launch(const SkinnyPlan& plan, int64_t b, int m, int64_t k, i
 }
 
 cudaError_t skinny_reduce_launch(const float* partial, float* C, int64_t b, int m, int64_t n,
-                                 int64_t c_batch, int split_k, cudaStream_t stream) {
+                                 int64_t c_batch, int split_k, cudaStream_t stream, bool overwrite) {
   const int64_t total = b * m * n;
   const int64_t blocks = (total + 255) / 256;
   return launch_pdl(reduce_kernel, dim3((unsigned)blocks, 1, 1), 256, 0, stream, partial, C, total,
-                    (int64_t)m * n, c_batch, split_k);
+                    (int64_t)m * n, c_batch, split_k, overwrite ? 1 : 0);
 }
 
 }  // namespace morello

@@ -190,6 +190,29 @@ def test_accumulates_across_calls():
     assert_bit_exact(gpu_run(A, B, C, calls=3), thrice, "three accumulating calls")
 
 
+def test_back_to_back_calls_of_every_kernel_family_on_shared_buffers():
+    """Calls are launched so that each may start while its predecessor drains; a chain that
+    alternates kernel families on the same C (and re-uses one call's inputs in the next)
+    must still equal the oracle applied in order.  Integer inputs: every call is exact."""
+    b, k, n = 1, 512, 2048
+    rows = [1, 16, 1, 160, 2, 40, 1, 300, 16, 1]          # GEMV, swapped, tiles, pairs, ...
+    m_max = max(rows)
+    A, B, C = w.make(b, m_max, k, n, seed=31, ab="int4", c="int8")
+    B2 = w.make(b, 1, k, n, seed=32, ab="int4", c="zeros")[1]
+    dA, dB, dC = to_dev(A, B, C)
+    dB2 = torch.from_numpy(B2.view(np.int16)).cuda()
+    want = C.copy()
+    for step, m in enumerate(rows):
+        Bs, dBs = (B, dB) if step % 2 == 0 else (B2, dB2)
+        # rows [0, m) of A against C's first m rows: a sub-problem with the same row pitch
+        mb.morello_matmul_accum(b, m, k, n, dA, dBs, dC)
+        want[:, :m, :] = oracle.matmul_accum(b, m, k, n, np.ascontiguousarray(A[:, :m, :]), Bs,
+                                             np.ascontiguousarray(want[:, :m, :]))
+    st, detail = mb.morello_read_device_status()
+    assert st == mb.MORELLO_OK, hex(detail)
+    assert_bit_exact(dC.cpu().numpy(), want, "chain of calls on one C")
+
+
 # ------------------------------------------------------------------ T5: guards
 def test_canaries_around_c_stay_intact():
     b, m, k, n = 2, 5, 96, 40
