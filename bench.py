@@ -235,7 +235,7 @@ def time_calls(torch, fn, steps, warmup):
     return start.elapsed_time(stop) * 1e-3
 
 
-def bench_config(torch, mb, idx, iters, warmup, peaks, windows, path=None, split_k=0):
+def bench_config(torch, mb, idx, iters, warmup, peaks, windows, path=None, split_k=0, op="matmul_accum"):
     """Device-timed throughput of one config (inputs resident, rotating when small)."""
     cfg = w.CONFIGS[idx]
     b, m, k, n = cfg.shape
@@ -252,7 +252,7 @@ def bench_config(torch, mb, idx, iters, warmup, peaks, windows, path=None, split
                     torch.from_numpy(C.copy()).cuda()))
     ptrs = [(a.data_ptr(), bb.data_ptr(), c.data_ptr()) for (a, bb, c) in dev]
     stream = torch.cuda.current_stream().cuda_stream
-    call = mb.lib().morello_matmul_accum_forced
+    call = mb.lib().morello_matmul_accum_forced if op == "matmul_accum" else mb.lib().morello_matmul_forced
     forced = mb.MORELLO_PATH_AUTO if path is None else path
 
     def step(i):
@@ -271,10 +271,11 @@ def bench_config(torch, mb, idx, iters, warmup, peaks, windows, path=None, split
     if st != 0:
         raise RuntimeError("device status %d (0x%x) after %s" % (st, detail, cfg.name))
     us = sec / iters * 1e6
-    gbs = cfg.algorithmic_bytes / (sec / iters) / 1e9
+    alg_bytes = cfg.algorithmic_bytes - (4 * b * m * n if op == "matmul" else 0)   # Matmul never reads C
+    gbs = alg_bytes / (sec / iters) / 1e9
     tfl = cfg.flops / (sec / iters) / 1e12
     chosen = mb.morello_select_path(b, m, k, n) if path is None else path
-    rec = {"name": cfg.name, "shape": list(cfg.shape), "path": "tcgen05" if chosen == 1 else "skinny",
+    rec = {"name": cfg.name, "op": op, "shape": list(cfg.shape), "path": "tcgen05" if chosen == 1 else "skinny",
            "us_per_call": us, "GBps": gbs, "TFLOPs": tfl, "iters": iters, "launches_per_call": per_call,
            "rotating_sets": sets,
            "frac_hbm_measured": gbs / peaks["hbm_gbs"], "frac_hbm_nominal": gbs / NOMINAL_HBM_GBS,
@@ -437,6 +438,8 @@ def run_ours(args):
                 continue
             iters, wu = plan[idx]
             extra.append(bench_config(torch, mb, idx, iters, wu, peaks, windows))
+            if idx == 4:                        # the large config also without the read of C (Matmul)
+                extra.append(bench_config(torch, mb, idx, iters, wu, peaks, windows, op="matmul"))
             if idx == 2:                        # crossover config: also on the path not chosen
                 other = (mb.MORELLO_PATH_TCGEN05
                          if mb.morello_select_path(*w.CONFIGS[2].shape) == mb.MORELLO_PATH_SKINNY
