@@ -220,6 +220,22 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------ GPU arm
+def max_over_ranks(seconds, dist, device):
+    """The slowest rank's time (replicas run independently; the job is as slow as its slowest
+    member).  `dist` is torch.distributed with an initialised process group, or None."""
+    if dist is None:
+        return float(seconds)
+    import torch
+    t = torch.tensor([seconds], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank_per_step, steps, world, seconds):
+    """Aggregate throughput of `world` replicas that each did `steps` steps in `seconds`."""
+    return world * units_per_rank_per_step * steps / seconds
+
+
 def time_calls(torch, fn, steps, warmup):
     """fn(i) enqueues step i on the current stream; returns seconds for `steps` steps."""
     for i in range(warmup):
@@ -368,14 +384,11 @@ def run_ours(args):
         torch.cuda.synchronize()
     launches = mb.morello_launch_count() - l0
     sec = start.elapsed_time(stop) * 1e-3
-    if dist is not None:
-        t = torch.tensor([sec], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        sec = float(t.item())
+    sec = max_over_ranks(sec, dist, "cuda")
     st, detail = mb.morello_read_device_status()
     if st != 0:
         raise RuntimeError("device status %d (0x%x)" % (st, detail))
-    value = world * cfg.algorithmic_bytes * args.steps / sec / 1e9
+    value = whole_job_value(cfg.algorithmic_bytes, args.steps, world, sec) / 1e9
 
     # ---- the same loop replayed from a CUDA graph (launch overhead taken out)
     graph_us = None
@@ -422,10 +435,7 @@ def run_ours(args):
         assert host_call(b, m, k, n, hA.data_ptr(), hB[i % 2].data_ptr(), hC.data_ptr()) == 0
     e2e_sec = time.perf_counter() - t0        # the call returns only when C is back on the host
     windows.append((t0, time.perf_counter()))
-    if dist is not None:
-        t = torch.tensor([e2e_sec], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_sec = float(t.item())
+    e2e_sec = max_over_ranks(e2e_sec, dist, "cuda")
     e2e_value = world * cfg.algorithmic_bytes * e2e_steps / e2e_sec / 1e9
     h2d = 2 * b * m * k + 2 * b * k * n + 4 * b * m * n
     d2h = 4 * b * m * n
