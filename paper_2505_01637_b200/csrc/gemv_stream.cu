@@ -3,15 +3,15 @@
 //
 // Decomposition.  The n columns are cut into strips of 64 (one 128-byte row segment of
 // bf16) and, when the strips alone cannot fill the device or k is long, the k range into
-// slices that are multiples of 64 rows.  One thread block owns one (batch, strip, slice):
-//   warp 0      producer: one lane walks the slice in boxes of 64 k rows x 64 columns
-//               (8 KiB), issuing TMA loads into a ring of shared-memory stages, each
+// slices that are multiples of 128 rows.  One thread block owns one (batch, strip, slice):
+//   warp 0      producer: one lane walks the slice in boxes of 128 k rows x 64 columns
+//               (16 KiB), issuing TMA loads into a ring of 5 shared-memory stages, each
 //               completing on the stage's "full" mbarrier;
 //   warps 1-8   consumers: a warp reads 4 rows x 128 bytes per 16-byte-per-lane load, widens
 //               bf16 to f32 (exact), multiplies by the rows' A values (the slice of A is
 //               brought into shared memory once, by bulk copies when its alignment allows)
-//               and accumulates 8 columns x m rows per lane; each warp then frees the stage
-//               on its "empty" mbarrier.
+//               and accumulates 8 columns x m rows per lane with packed f32x2 FMAs; each warp
+//               then frees the stage on its "empty" mbarrier.
 // At the end the four row groups of a warp are added with shuffles and the eight warps
 // through shared memory, always in the same order, so results are deterministic.  With one
 // slice the block adds its sums to C (C was read early, the addition happens once, last);
@@ -23,9 +23,9 @@
 // nothing into the SM and cannot observe stale data, so it is legal before the preceding
 // kernel has completed.  A block lets dependents launch when its producer has issued its
 // last load: the next call's blocks then arrive while this call drains, and their
-// prefetches keep HBM busy through this call's tail and the launch gap.  Blocks are small
-// enough (288 threads, about 55 KiB of shared memory for m = 1) for the next call's blocks
-// to be resident next to this call's.
+// prefetches keep HBM busy through this call's tail and the launch gap.  The ring (80 KiB)
+// is sized so that at most two blocks share an SM: with three, the blocks of the crowded SMs
+// finish microseconds after the rest.
 //
 // Rows of a box past k and columns past n are zero-filled by the TMA engine.  Every
 // barrier wait is bounded; on a timeout the block records a status word and writes nothing.
@@ -46,13 +46,19 @@ using namespace sm100;
 #define MORELLO_GEMV_STRIP_COLS 64
 #endif
 #ifndef MORELLO_GEMV_STAGES
-#define MORELLO_GEMV_STAGES 10
+#define MORELLO_GEMV_STAGES 5
 #endif
 #ifndef MORELLO_GEMV_PREFETCH_BOXES
-#define MORELLO_GEMV_PREFETCH_BOXES 12
+#define MORELLO_GEMV_PREFETCH_BOXES 6
 #endif
 constexpr int kStripCols = MORELLO_GEMV_STRIP_COLS;         // columns per thread block: 64 or 128
-constexpr int kBoxRows = 64;                                // k rows per stage
+#ifndef MORELLO_GEMV_BOX_ROWS
+#define MORELLO_GEMV_BOX_ROWS 128
+#endif
+#ifndef MORELLO_GEMV_FFMA2
+#define MORELLO_GEMV_FFMA2 1
+#endif
+constexpr int kBoxRows = MORELLO_GEMV_BOX_ROWS;             // k rows per stage: 64 or 128
 constexpr int kStageBytes = kBoxRows * kStripCols * 2;      // 8 or 16 KiB
 constexpr int kStages = MORELLO_GEMV_STAGES;
 constexpr int kConsumerWarps = 8;
@@ -95,6 +101,26 @@ __device__ __forceinline__ void consumer_sync() {
 }
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// Two f32 lanes in one 64-bit register, and acc = a * b + acc on both lanes at once
+// (fma.rn.f32x2: each lane is an ordinary round-to-nearest FMA, so results equal two fmaf).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void fma2(uint64_t& acc, uint64_t a, uint64_t b) {
+#if MORELLO_GEMV_FFMA2
+  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
+#else
+  float a0, a1, b0, b1, c0, c1;
+  unpack2(a, a0, a1); unpack2(b, b0, b1); unpack2(acc, c0, c1);
+  acc = pack2(fmaf(a0, b0, c0), fmaf(a1, b1, c1));
+#endif
+}
 
 template <int M_T>
 __global__ void __launch_bounds__(kThreads)
@@ -200,11 +226,11 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_b, const StreamParams
   }
   consumer_sync();
 
-  float acc[M_T][8];
+  uint64_t acc2[M_T][4];                  // columns (2h, 2h + 1) of the chunk, as f32 pairs
 #pragma unroll
   for (int i = 0; i < M_T; ++i)
 #pragma unroll
-    for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+    for (int h = 0; h < 4; ++h) acc2[i][h] = 0ull;
 
   bool ok = true;
   if (p.a_bulk) {
@@ -230,19 +256,18 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_b, const StreamParams
       const uint16_t* a_col = a_s + j * kBoxRows + row_in_box;
 #pragma unroll
       for (int u = 0; u < kPasses; ++u) {
-        float a[M_T];
+        uint64_t a2[M_T];                 // the row's multiplier on both lanes
 #pragma unroll
-        for (int i = 0; i < M_T; ++i)
-          a[i] = __uint_as_float(((uint32_t)a_col[(size_t)i * p.k_per_split + u * kRowsPerPass]) << 16);
+        for (int i = 0; i < M_T; ++i) {
+          const float a = __uint_as_float(((uint32_t)a_col[(size_t)i * p.k_per_split + u * kRowsPerPass]) << 16);
+          a2[i] = pack2(a, a);
+        }
         const uint32_t ww[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
 #pragma unroll
         for (int h = 0; h < 4; ++h) {
-          const float lo = bf16_lo(ww[h]), hi = bf16_hi(ww[h]);
+          const uint64_t b2 = pack2(bf16_lo(ww[h]), bf16_hi(ww[h]));
 #pragma unroll
-          for (int i = 0; i < M_T; ++i) {
-            acc[i][2 * h] = fmaf(a[i], lo, acc[i][2 * h]);
-            acc[i][2 * h + 1] = fmaf(a[i], hi, acc[i][2 * h + 1]);
-          }
+          for (int i = 0; i < M_T; ++i) fma2(acc2[i][h], a2[i], b2);
         }
       }
       __syncwarp();                       // every lane's reads of the stage are done
@@ -251,6 +276,11 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_b, const StreamParams
     }
   }
 
+  float acc[M_T][8];
+#pragma unroll
+  for (int i = 0; i < M_T; ++i)
+#pragma unroll
+    for (int h = 0; h < 4; ++h) unpack2(acc2[i][h], acc[i][2 * h], acc[i][2 * h + 1]);
   // Row groups of the warp, pairwise, in the same order in every lane.
 #pragma unroll
   for (int i = 0; i < M_T; ++i)
