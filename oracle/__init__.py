@@ -48,6 +48,8 @@ def _load():
         lib.oracle_matmul_accum_rows.restype = ctypes.c_int
         lib.oracle_abs_dot.argtypes = [i64, i64, i64, i64, vp, vp, vp]
         lib.oracle_abs_dot.restype = None
+        lib.oracle_matmul_accum_f32.argtypes = [i64, i64, i64, i64, vp, vp, vp, vp]
+        lib.oracle_matmul_accum_f32.restype = ctypes.c_int
         lib.oracle_num_threads.restype = ctypes.c_int
         lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
         _lib = lib
@@ -100,6 +102,18 @@ def abs_dot(b, m, k, n, A, B) -> np.ndarray:
     T = np.zeros((b, m, n), dtype=np.float64)
     _load().oracle_abs_dot(b, m, k, n, _ptr(A), _ptr(B), _ptr(T))
     return T
+
+
+def matmul_accum_f32(b, m, k, n, A, B, C, want_abs: bool = False):
+    """float32 inputs: returns C + A x B (new f32 array), and sum_p |A*B| (f64) if asked."""
+    for x, size in ((A, b * m * k), (B, b * k * n), (C, b * m * n)):
+        assert x.dtype == np.float32 and x.flags.c_contiguous and x.size == size
+    out = np.array(C, dtype=np.float32, copy=True, order="C")
+    T = np.zeros((b, m, n), dtype=np.float64) if want_abs else None
+    rc = _load().oracle_matmul_accum_f32(b, m, k, n, _ptr(A), _ptr(B), _ptr(out), _ptr(T))
+    if rc != 0:
+        raise MemoryError("oracle scratch allocation failed")
+    return (out, T) if want_abs else out
 
 
 def num_threads() -> int:

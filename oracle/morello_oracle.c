@@ -191,3 +191,47 @@ void oracle_set_num_threads(int t) { if (t > 0) omp_set_num_threads(t); }
 int oracle_num_threads(void) { return 1; }
 void oracle_set_num_threads(int t) { (void)t; }
 #endif
+
+/*
+ * The same operation on float32 inputs (the paper's other benchmark, Section 7: a
+ * float32, 2048-square matrix multiplication):
+ *
+ *     C[b,i,j]  <-  C[b,i,j] + sum_{p=0}^{k-1} A[b,i,p] * B[b,p,j],   A, B, C float
+ *
+ * A product of two floats has at most 48 significant bits and is exact in double; the
+ * sum starts from (double)C, runs over p in increasing order in double and is rounded
+ * once to float.  T (may be NULL) receives sum_p |A*B|.  Rows are independent and are
+ * handed to host threads.  Returns 0, or -1 if a row buffer could not be allocated.
+ */
+int oracle_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n,
+                            const float *A, const float *B, float *C, double *T)
+{
+    if (b <= 0 || m <= 0 || n <= 0) return 0;
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *s = (double *)malloc((size_t)n * sizeof(double));
+        if (!s) {
+#pragma omp atomic write
+            failed = 1;
+        } else {
+#pragma omp for schedule(dynamic, 1)
+            for (int64_t r = 0; r < b * m; ++r) {
+                const int64_t bb = r / m;
+                float *Crow = C + r * n;
+                double *Trow = T ? T + r * n : NULL;
+                for (int64_t j = 0; j < n; ++j) s[j] = (double)Crow[j];
+                if (Trow) for (int64_t j = 0; j < n; ++j) Trow[j] = 0.0;
+                for (int64_t p = 0; p < k; ++p) {
+                    const double a = (double)A[r * k + p];
+                    const float *Brow = B + (bb * k + p) * n;
+                    for (int64_t j = 0; j < n; ++j) s[j] += a * (double)Brow[j];
+                    if (Trow) for (int64_t j = 0; j < n; ++j) Trow[j] += fabs(a * (double)Brow[j]);
+                }
+                for (int64_t j = 0; j < n; ++j) Crow[j] = (float)s[j];
+            }
+        }
+        free(s);
+    }
+    return failed ? -1 : 0;
+}

@@ -320,3 +320,70 @@ def test_pins_detect_planted_mistakes(kind):
     want = exact_matmul_accum_bits(A, B, C)
     assert np.array_equal(bits(run(A, B, C)), want)
     assert not np.array_equal(bits(_mutant(A, B, C, kind)), want)
+
+
+# ---------------------------------------------------- float32-input oracle (Section 7's
+# float32 2048-square matmul): pinned to the bf16 oracle above, to exact rational
+# arithmetic and to layout one-hots
+def exact_f32_bits(A, B, C):
+    b, m, k = A.shape
+    n = B.shape[2]
+    out = np.zeros((b, m, n), dtype=np.uint32)
+    for bb in range(b):
+        for i in range(m):
+            for j in range(n):
+                s = Fraction(float(C[bb, i, j]))
+                for p in range(k):
+                    s += Fraction(float(A[bb, i, p])) * Fraction(float(B[bb, p, j]))
+                out[bb, i, j] = frac_to_f32_bits(s)
+    return out
+
+
+def test_f32_oracle_equals_bf16_oracle_on_bf16_representable_inputs():
+    for (b, m, k, n) in [(1, 4, 4, 16), (2, 3, 65, 40), (1, 1, 257, 33)]:
+        A, B, C = w.make(b, m, k, n, seed=3 + k, ab="uniform", c="normal")
+        want = oracle.matmul_accum(b, m, k, n, A, B, C)
+        got = oracle.matmul_accum_f32(b, m, k, n, w.bf16_to_f32(A), w.bf16_to_f32(B), C)
+        assert np.array_equal(bits(got), bits(want))
+
+
+@pytest.mark.parametrize("shape", [(1, 1, 1, 1), (2, 3, 5, 7), (1, 4, 9, 3)])
+def test_f32_oracle_exact_rational_brute_force(shape):
+    b, m, k, n = shape
+    rng = np.random.Generator(np.random.Philox(40 + sum(shape)))
+    # 12 significant bits per input: products have 24, and sums of a few of them are exact in
+    # double, so the oracle's single rounding must equal the exact result's rounding
+    def q12(x):
+        mant, ex = np.frexp(x.astype(np.float64))
+        return np.ldexp(np.round(mant * 4096) / 4096, ex).astype(np.float32)
+    A = q12(rng.standard_normal((b, m, k)))
+    B = q12(rng.standard_normal((b, k, n)))
+    C = q12(rng.standard_normal((b, m, n)))
+    got = oracle.matmul_accum_f32(b, m, k, n, A, B, C)
+    assert np.array_equal(bits(got), exact_f32_bits(A, B, C))
+    # full-precision inputs: the double sum may round once more than the exact one; never
+    # further than one unit in the last place
+    A = rng.standard_normal((b, m, k)).astype(np.float32)
+    B = rng.standard_normal((b, k, n)).astype(np.float32)
+    C = rng.standard_normal((b, m, n)).astype(np.float32)
+    got = bits(oracle.matmul_accum_f32(b, m, k, n, A, B, C)).astype(np.int64)
+    want = exact_f32_bits(A, B, C).astype(np.int64)
+    assert np.abs(got - want).max() <= 1
+
+
+def test_f32_oracle_one_hot_layout_abs_dot_and_float64_agreement():
+    b, m, k, n = 3, 4, 6, 5
+    rng = np.random.default_rng(5)
+    Bv = rng.integers(-100, 101, size=(b, k, n)).astype(np.float32)
+    C = rng.integers(-50, 51, size=(b, m, n)).astype(np.float32)
+    A1 = np.zeros((b, m, k), np.float32)
+    A1[1, 2, 4] = 2.0
+    want = C.copy()
+    want[1, 2, :] += 2.0 * Bv[1, 4, :]
+    assert np.array_equal(oracle.matmul_accum_f32(b, m, k, n, A1, Bv, C), want)
+    A = rng.standard_normal((b, m, k)).astype(np.float32)
+    B = rng.standard_normal((b, k, n)).astype(np.float32)
+    got, T = oracle.matmul_accum_f32(b, m, k, n, A, B, C, want_abs=True)
+    ref = C.astype(np.float64) + np.einsum("bik,bkj->bij", A.astype(np.float64), B.astype(np.float64))
+    assert np.abs(got - ref).max() <= np.spacing(np.abs(ref).max().astype(np.float32))
+    assert np.allclose(T, np.einsum("bik,bkj->bij", np.abs(A).astype(np.float64), np.abs(B).astype(np.float64)), rtol=1e-12)
