@@ -110,6 +110,23 @@ int morello_matmul_forced(int path, int split_k,
                           void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * MatmulAccum on float32 inputs (the paper's other benchmark, Section 7, is a float32
+ * 2048-square matrix multiplication): A[b][m][k], B[b][k][n] and C[b][m][n] all f32, dense
+ * row-major device pointers, 4-byte aligned; C += A x B.
+ * Each float is split exactly into three bf16 terms and the six largest of the nine cross
+ * products are computed by the bf16 kernels in one MatmulAccum(b, m, 6k, n) (the dropped
+ * terms are below 2^-23 of |a*b|), so the result meets the same acceptance rule as the bf16
+ * operation, is deterministic, and is exact when the inputs are bf16-representable.  The
+ * split operands (12 bytes per element of A and B) live in a per-device buffer owned by
+ * the library that grows on demand (the call may allocate, and synchronises the device when
+ * it has to grow the buffer); concurrent calls on different streams share that buffer and
+ * must be serialised by the caller.  Meant for GEMM-shaped problems: with few rows the
+ * split of B costs more than the multiply.  Finite inputs only.
+ */
+int morello_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n,
+                             const float* A, const float* B, float* C, void* stream);
+
+/*
  * End-to-end convenience call on HOST buffers (same layouts): copies A, B and
  * C to library-owned device staging (grown on demand), runs the operation,
  * copies C back and synchronises before returning.  Pinned host memory makes

@@ -21,6 +21,8 @@ struct DeviceState {
   size_t scratch_bytes = 0;
   void* stage = nullptr;         // device staging for the host-buffer entry point
   size_t stage_bytes = 0;
+  void* split = nullptr;         // bf16 terms of float32 operands (morello_matmul_accum_f32)
+  size_t split_bytes = 0;
 };
 
 std::mutex g_mutex;
@@ -296,6 +298,52 @@ int morello_matmul_forced(int path, int split_k, int64_t b, int64_t m, int64_t k
                           size_t workspace_bytes, void* stream) {
   const bool own = (workspace == nullptr && workspace_bytes == 0);
   return run(path, split_k, b, m, k, n, A, B, C, workspace, workspace_bytes, own, stream, true);
+}
+
+int morello_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n, const float* A,
+                             const float* B, float* C, void* stream) {
+  if (b < 0 || m < 0 || k < 0 || n < 0) return MORELLO_ERR_INVALID_SHAPE;
+  int64_t k6, t;
+  if (mul_overflows(k, 6, &k6) || mul_overflows(m, k6, &t) || mul_overflows(b, t, &t) ||
+      mul_overflows(t, 2, &t) || mul_overflows(k6, n, &t) || mul_overflows(b, t, &t) ||
+      mul_overflows(t, 2, &t))
+    return MORELLO_ERR_INVALID_SHAPE;
+  bool empty = false;
+  // Shape, null and alignment checks of the bf16 problem the call turns into, with the
+  // float pointers standing in (4-byte alignment is what they need).
+  int rc = validate(b, m, k6, n, A, B, C, &empty);
+  if (rc != MORELLO_OK) return rc;
+  if (!empty && (reinterpret_cast<uintptr_t>(A) % 4 || reinterpret_cast<uintptr_t>(B) % 4))
+    return MORELLO_ERR_MISALIGNED;
+  DeviceState* st = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    rc = device_state(&st);
+  }
+  if (rc != MORELLO_OK || empty) return rc;
+  const size_t need = f32_split_bytes(b, m, k, n);
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (st->split_bytes < need) {
+      cudaError_t e = cudaDeviceSynchronize();   // work in flight may still read the old buffer
+      if (e != cudaSuccess) return cuda_fail(e);
+      if (st->split) cudaFree(st->split);
+      st->split = nullptr;
+      st->split_bytes = 0;
+      if ((e = cudaMalloc(&st->split, need)) != cudaSuccess) {
+        cuda_fail(e);
+        return MORELLO_ERR_WORKSPACE;
+      }
+      st->split_bytes = need;
+    }
+  }
+  uint16_t *A6 = nullptr, *B6 = nullptr;
+  uint64_t launches = 0;
+  const cudaError_t e = f32_split_launch(b, m, k, n, A, B, st->split, &A6, &B6,
+                                         static_cast<cudaStream_t>(stream), &launches);
+  g_launches.fetch_add(launches, std::memory_order_relaxed);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return run(MORELLO_PATH_AUTO, 0, b, m, k6, n, A6, B6, C, nullptr, 0, true, stream);
 }
 
 int morello_matmul_accum_host(int64_t b, int64_t m, int64_t k, int64_t n, const void* A_host,

@@ -1,0 +1,88 @@
+// MatmulAccum on float32 inputs through the bf16 tensor-core kernels.
+//
+// A float is the exact sum of three bf16 values: x1 = bf16(x), x2 = bf16(x - x1),
+// x3 = bf16(x - x1 - x2) (each difference is exact in float: every bf16 takes the next 8 of
+// the 24 significant bits).  Then
+//     a * b = sum over i, j of a_i * b_j,
+// where a_i * b_j is about 2^(-8 (i + j - 2)) of a * b.  The six terms with i + j <= 4 are
+// kept; the three dropped ones are below 2^-23 of |a * b|, well inside the acceptance rule
+// (1e-5 of sum |a * b|).  Each kept term is a bf16 x bf16 product, exact in f32, which is
+// what the tensor-core kernels accumulate.
+//
+// Rather than six calls, the six terms are laid side by side along k: the split kernels write
+//     A6[b][m][6k] = [ A3 | A1 | A2 | A2 | A1 | A1 ]        (columns)
+//     B6[b][6k][n] = [ B1 ; B3 ; B2 ; B1 ; B2 ; B1 ]        (rows)
+// so that A6 x B6 = A3 B1 + A1 B3 + A2 B2 + A2 B1 + A1 B2 + A1 B1 (smallest terms first), and
+// one ordinary MatmulAccum(b, m, 6k, n) on bf16 does the rest -- same kernels, same selector,
+// C added once, deterministic.  Inputs whose values are bf16-exact (small integers, say) give
+// A2 = A3 = 0 and the result is exact.
+#include "internal.h"
+
+namespace morello {
+namespace {
+
+__device__ __forceinline__ uint16_t bf16_rne(float x) {   // finite inputs
+  const uint32_t u = __float_as_uint(x);
+  return (uint16_t)((u + 0x7fffu + ((u >> 16) & 1u)) >> 16);
+}
+__device__ __forceinline__ float bf16_as_float(uint16_t h) { return __uint_as_float(((uint32_t)h) << 16); }
+
+__device__ __forceinline__ void split3(float x, uint16_t& h1, uint16_t& h2, uint16_t& h3) {
+  h1 = bf16_rne(x);
+  const float r1 = x - bf16_as_float(h1);       // exact
+  h2 = bf16_rne(r1);
+  const float r2 = r1 - bf16_as_float(h2);      // exact
+  h3 = bf16_rne(r2);
+}
+
+// A[rows][k] -> A6[rows][6k], blocks of k columns in the order 3, 1, 2, 2, 1, 1.
+__global__ void __launch_bounds__(256)
+split_a_kernel(const float* __restrict__ A, uint16_t* __restrict__ A6, int64_t rows, int64_t k) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= rows * k) return;
+  const int64_t r = idx / k, p = idx - r * k;
+  uint16_t h1, h2, h3;
+  split3(A[idx], h1, h2, h3);
+  uint16_t* row = A6 + r * 6 * k + p;
+  row[0] = h3; row[k] = h1; row[2 * k] = h2; row[3 * k] = h2; row[4 * k] = h1; row[5 * k] = h1;
+}
+
+// B[b][k][n] -> B6[b][6k][n], blocks of k rows in the order 1, 3, 2, 1, 2, 1.
+__global__ void __launch_bounds__(256)
+split_b_kernel(const float* __restrict__ B, uint16_t* __restrict__ B6, int64_t b, int64_t k, int64_t n) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= b * k * n) return;
+  const int64_t kn = k * n;
+  const int64_t bb = idx / kn, rest = idx - bb * kn;      // rest = p * n + j
+  uint16_t h1, h2, h3;
+  split3(B[idx], h1, h2, h3);
+  uint16_t* dst = B6 + bb * 6 * kn + rest;
+  dst[0] = h1; dst[kn] = h3; dst[2 * kn] = h2; dst[3 * kn] = h1; dst[4 * kn] = h2; dst[5 * kn] = h1;
+}
+
+}  // namespace
+
+size_t f32_split_bytes(int64_t b, int64_t m, int64_t k, int64_t n) {
+  auto round256 = [](size_t x) { return (x + 255) / 256 * 256; };
+  return round256((size_t)b * m * k * 12) + round256((size_t)b * k * n * 12);
+}
+
+cudaError_t f32_split_launch(int64_t b, int64_t m, int64_t k, int64_t n, const float* A, const float* B,
+                             void* split, uint16_t** A6, uint16_t** B6, cudaStream_t stream,
+                             uint64_t* launches) {
+  auto round256 = [](size_t x) { return (x + 255) / 256 * 256; };
+  *A6 = static_cast<uint16_t*>(split);
+  *B6 = reinterpret_cast<uint16_t*>(static_cast<char*>(split) + round256((size_t)b * m * k * 12));
+  const int64_t ea = b * m * k, eb = b * k * n;
+  split_a_kernel<<<(unsigned)((ea + 255) / 256), 256, 0, stream>>>(A, *A6, b * m, k);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  ++*launches;
+  split_b_kernel<<<(unsigned)((eb + 255) / 256), 256, 0, stream>>>(B, *B6, b, k, n);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  ++*launches;
+  return cudaSuccess;
+}
+
+}  // namespace morello

@@ -70,6 +70,14 @@ cudaError_t stream_launch(const DeviceInfo& dev, const StreamPlan& plan, int64_t
                           int64_t c_batch, float* workspace, cudaStream_t stream,
                           uint64_t* launches, bool overwrite = false);
 
+// ---- float32 inputs: split into bf16 terms laid side by side along k ----------
+// Bytes of the buffer that holds A6[b][m][6k] and B6[b][6k][n] (bf16).
+size_t f32_split_bytes(int64_t b, int64_t m, int64_t k, int64_t n);
+// Enqueues the two split kernels; *A6 and *B6 point into `split` afterwards.
+cudaError_t f32_split_launch(int64_t b, int64_t m, int64_t k, int64_t n, const float* A, const float* B,
+                             void* split, uint16_t** A6, uint16_t** B6, cudaStream_t stream,
+                             uint64_t* launches);
+
 // ---- tcgen05 path ------------------------------------------------------------
 struct GemmPlan {
   bool supported;
