@@ -338,6 +338,43 @@ def bench_f32_square(torch, mb, peaks, windows, size=2048, iters=20):
             "note": "inputs split exactly into three bf16 terms; six of nine cross products kept"}
 
 
+def bench_colmajor(torch, mb, idx, iters, peaks, windows):
+    """A config with its B stored column-major (Bt[b][n][k]) through
+    morello_matmul_accum_colmajor_b; inputs rotate like bench_config's."""
+    cfg = w.CONFIGS[idx]
+    b, m, k, n = cfg.shape
+    in_bytes = 2 * b * m * k + 2 * b * k * n + 4 * b * m * n
+    sets = max(1, min(ROTATE, int(np.ceil(512 * 2 ** 20 / in_bytes))))
+    dev = []
+    for s_ in range(sets):
+        As, Bs, Cs = w.make(b, m, k, n, 1000 * idx + 100 * s_ + 50, cfg.ab, "zeros")
+        Bt = np.ascontiguousarray(Bs.transpose(0, 2, 1))
+        dev.append((torch.from_numpy(As.view(np.int16)).cuda(), torch.from_numpy(Bt.view(np.int16)).cuda(),
+                    torch.from_numpy(Cs).cuda()))
+    ptrs = [(a.data_ptr(), bb.data_ptr(), c.data_ptr()) for (a, bb, c) in dev]
+    stream = torch.cuda.current_stream().cuda_stream
+    call = mb.lib().morello_matmul_accum_colmajor_b
+
+    def step(i):
+        pa, pb, pc = ptrs[i % sets]
+        rc = call(0, b, m, k, n, pa, pb, pc, stream)
+        if rc != 0:
+            raise mb.MorelloError(rc, "bench col-major %s" % cfg.name)
+
+    l0 = mb.morello_launch_count()
+    step(0)
+    per_call = mb.morello_launch_count() - l0
+    t0 = time.perf_counter()
+    loops = [time_calls(torch, step, iters, 5 if r == 0 else 3) for r in range(3)]
+    windows.append((t0, time.perf_counter()))
+    sec = min(loops) / iters
+    return {"name": cfg.name, "op": "matmul_accum_colmajor_b", "shape": list(cfg.shape), "path": "tcgen05",
+            "us_per_call": sec * 1e6, "GBps": cfg.algorithmic_bytes / sec / 1e9, "TFLOPs": cfg.flops / sec / 1e12,
+            "iters": iters, "launches_per_call": per_call, "rotating_sets": sets,
+            "frac_hbm_measured": cfg.algorithmic_bytes / sec / 1e9 / peaks["hbm_gbs"],
+            "frac_tensor_measured_burst": cfg.flops / sec / 1e12 / peaks["bf16_tflops"]}
+
+
 def run_case(args):
     """One configuration alone, device-timed: the command the ncu captures under
     profiles/ were taken with, and the unit of the sweeps quoted in the design notes."""
@@ -495,6 +532,9 @@ def run_ours(args):
                     pass
     if world == 1 and args.configs:
         extra.append(bench_f32_square(torch, mb, peaks, windows))
+        extra.append(bench_colmajor(torch, mb, HEADLINE, 300, peaks, windows))
+        if 3 in args.configs:
+            extra.append(bench_colmajor(torch, mb, 3, 30, peaks, windows))
     sampler.stop()
     clocks = sampler.summary(windows)
 

@@ -110,6 +110,21 @@ int morello_matmul_forced(int path, int split_k,
                           void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * MatmulAccum with B stored column-major (layouts are a field of the paper's Spec; its
+ * example in Section 2.2, a 1x4x128x16 Matmul, has a col_major right-hand side):
+ *
+ *     C[b,i,j]  <-  C[b,i,j] + sum_{p<k} A[b,i,p] * Bt[b,j,p],    Bt[b][n][k] bf16, k contiguous
+ *
+ * A and C as everywhere else.  With k % 8 == 0, n % 8 == 0 and 16-byte-aligned pointers the
+ * tensor-core kernels run it (for them a column-major B is the K-major operand; `tile` is
+ * their tile selector as in morello_matmul_accum_forced, 0 = by shape); any other shape
+ * runs on a plain one-warp-per-column kernel.  No scratch, no allocation.  Same status
+ * codes, asynchronous on `stream`, deterministic.
+ */
+int morello_matmul_accum_colmajor_b(int tile, int64_t b, int64_t m, int64_t k, int64_t n,
+                                    const void* A, const void* Bt, float* C, void* stream);
+
+/*
  * MatmulAccum on float32 inputs (the paper's other benchmark, Section 7, is a float32
  * 2048-square matrix multiplication): A[b][m][k], B[b][k][n] and C[b][m][n] all f32, dense
  * row-major device pointers, 4-byte aligned; C += A x B.

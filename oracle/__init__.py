@@ -50,6 +50,8 @@ def _load():
         lib.oracle_abs_dot.restype = None
         lib.oracle_matmul_accum_f32.argtypes = [i64, i64, i64, i64, vp, vp, vp, vp]
         lib.oracle_matmul_accum_f32.restype = ctypes.c_int
+        lib.oracle_matmul_accum_bt.argtypes = [i64, i64, i64, i64, vp, vp, vp]
+        lib.oracle_matmul_accum_bt.restype = None
         lib.oracle_num_threads.restype = ctypes.c_int
         lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
         _lib = lib
@@ -114,6 +116,16 @@ def matmul_accum_f32(b, m, k, n, A, B, C, want_abs: bool = False):
     if rc != 0:
         raise MemoryError("oracle scratch allocation failed")
     return (out, T) if want_abs else out
+
+
+def matmul_accum_bt(b, m, k, n, A, Bt, C) -> np.ndarray:
+    """B given column-major (Bt[b][n][k], bf16 bit patterns): returns C + A x B."""
+    assert Bt.dtype == np.uint16 and Bt.flags.c_contiguous and Bt.size == b * n * k
+    assert A.dtype == np.uint16 and A.flags.c_contiguous and A.size == b * m * k
+    out = np.array(C, dtype=np.float32, copy=True, order="C")
+    assert out.size == b * m * n
+    _load().oracle_matmul_accum_bt(b, m, k, n, _ptr(A), _ptr(Bt), _ptr(out))
+    return out
 
 
 def num_threads() -> int:

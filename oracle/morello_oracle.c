@@ -235,3 +235,28 @@ int oracle_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n,
     }
     return failed ? -1 : 0;
 }
+
+/*
+ * The bf16 operation with the right-hand side stored column-major (the paper's Spec
+ * carries a layout per operand; its Section 2.2 example has a col_major rhs):
+ *
+ *     C[b,i,j]  <-  C[b,i,j] + sum_{p=0}^{k-1} A[b,i,p] * Bt[b,j,p],   Bt[b][n][k]
+ *
+ * Same arithmetic as above (double accumulation of exact products in increasing p, one
+ * rounding); only the indexing of the right-hand side differs.
+ */
+void oracle_matmul_accum_bt(int64_t b, int64_t m, int64_t k, int64_t n,
+                            const uint16_t *A, const uint16_t *Bt, float *C)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < b * m; ++r) {
+        const int64_t bb = r / m;
+        for (int64_t j = 0; j < n; ++j) {
+            double s = (double)C[r * n + j];
+            const uint16_t *col = Bt + (bb * n + j) * k;
+            for (int64_t p = 0; p < k; ++p)
+                s += bf16_to_double(A[r * k + p]) * bf16_to_double(col[p]);
+            C[r * n + j] = (float)s;
+        }
+    }
+}

@@ -150,7 +150,7 @@ size_t workspace_for(int sms, int path, int knob, int64_t b, int64_t m, int64_t 
 
 int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
         const void* B, float* C, void* workspace, size_t workspace_bytes, bool own_scratch,
-        void* stream, bool overwrite = false) {
+        void* stream, bool overwrite = false, bool b_col_major = false) {
   bool empty = false;
   int rc = validate(b, m, k, n, A, B, C, &empty);
   if (rc != MORELLO_OK) return rc;
@@ -174,6 +174,28 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     return MORELLO_OK;
   }
 
+  if (b_col_major) {
+    // B as [b][n][k]: the tensor-core kernels when the TMA engine can address the operands,
+    // else the one-warp-per-column kernel.  The FMA streaming kernels read B by rows only.
+    if (path == MORELLO_PATH_SKINNY) return MORELLO_ERR_UNSUPPORTED_PATH;
+    const bool tc = gemm_shape_supported(b, m, k, n, A, B, C);
+    if (path == MORELLO_PATH_TCGEN05 && !tc) return MORELLO_ERR_UNSUPPORTED_PATH;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint64_t launches = 0;
+    cudaError_t e;
+    if (tc) {
+      const GemmPlan plan = gemm_plan(st->info.sms, b, m, k, n, split_k);
+      if (!plan.supported) return MORELLO_ERR_UNSUPPORTED_PATH;
+      e = gemm_launch(st->info, plan, b, m, k, n, static_cast<const uint16_t*>(A),
+                      static_cast<const uint16_t*>(B), C, nullptr, s, &launches, overwrite, true);
+    } else {
+      e = colmajor_fallback_launch(b, m, k, n, static_cast<const uint16_t*>(A),
+                                   static_cast<const uint16_t*>(B), C, overwrite, s, &launches);
+    }
+    g_launches.fetch_add(launches, std::memory_order_relaxed);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return MORELLO_OK;
+  }
   if (path == MORELLO_PATH_AUTO) {
     path = select_path(st->info.sms, b, m, k, n, A, B, C);
   } else if (path == MORELLO_PATH_TCGEN05) {
@@ -298,6 +320,12 @@ int morello_matmul_forced(int path, int split_k, int64_t b, int64_t m, int64_t k
                           size_t workspace_bytes, void* stream) {
   const bool own = (workspace == nullptr && workspace_bytes == 0);
   return run(path, split_k, b, m, k, n, A, B, C, workspace, workspace_bytes, own, stream, true);
+}
+
+int morello_matmul_accum_colmajor_b(int tile, int64_t b, int64_t m, int64_t k, int64_t n,
+                                    const void* A, const void* Bt, float* C, void* stream) {
+  if (tile < 0) return MORELLO_ERR_INVALID_SHAPE;
+  return run(MORELLO_PATH_AUTO, tile, b, m, k, n, A, Bt, C, nullptr, 0, true, stream, false, true);
 }
 
 int morello_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n, const float* A,

@@ -81,6 +81,7 @@ struct GemmParams {
   int k_blocks;
   uint32_t* status;
   int overwrite;   // 1: C = product (TMA store) instead of C += product (TMA reduce-add)
+  int bt;          // 1: B is stored column-major, [b][n][k]: the K-major operand (boxes of 64 k x 64 columns)
   int a_box_rows;  // rows of A one TMA box brings: 128, or m rounded up to 16 when m < 128
 };
 
@@ -213,16 +214,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             tma_load_3d_pair(sa, &map_a, full, kb * kTileK, row0, bb);
 #pragma unroll
             for (int j = 0; j < S::kBoxesB; ++j)
-              if (j < boxes_b)
-                tma_load_3d_pair(sb + j * kBoxBytesB, &map_b, full, col0 + j * 64, kb * kTileK, bb);
+              if (j < boxes_b) {
+                if (p.bt) tma_load_3d_pair(sb + j * kBoxBytesB, &map_b, full, kb * kTileK, col0 + j * 64, bb);
+                else tma_load_3d_pair(sb + j * kBoxBytesB, &map_b, full, col0 + j * 64, kb * kTileK, bb);
+              }
           } else {
             mbar_arrive_expect_tx(&bars->full[stage], stage_tx);
             tma_load_3d(sa, &map_a, &bars->full[stage], kb * kTileK, row0, bb);
 #pragma unroll
             for (int j = 0; j < S::kBoxesB; ++j)
-              if (j < boxes_b)
-                tma_load_3d(sb + j * kBoxBytesB, &map_b, &bars->full[stage], col0 + j * 64,
-                            kb * kTileK, bb);
+              if (j < boxes_b) {
+                if (p.bt) tma_load_3d(sb + j * kBoxBytesB, &map_b, &bars->full[stage], kb * kTileK,
+                                      col0 + j * 64, bb);
+                else tma_load_3d(sb + j * kBoxBytesB, &map_b, &bars->full[stage], col0 + j * 64,
+                                 kb * kTileK, bb);
+              }
           }
           if (++stage == S::kStages) { stage = 0; phase ^= 1; }
         }
@@ -231,8 +237,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (rank == 0 && elect_one()) {
-      constexpr uint32_t idesc_tile = instr_desc_bf16(S::kTileM, kTileN, false, true);
-      constexpr uint32_t idesc_half = instr_desc_bf16(S::kTileM, kTileN / 2, false, true);
+      // B row-major is the MN-major operand, B column-major the K-major one.
+      const uint32_t idesc_tile = p.bt ? instr_desc_bf16(S::kTileM, kTileN, false, false)
+                                       : instr_desc_bf16(S::kTileM, kTileN, false, true);
+      const uint32_t idesc_half = p.bt ? instr_desc_bf16(S::kTileM, kTileN / 2, false, false)
+                                       : instr_desc_bf16(S::kTileM, kTileN / 2, false, true);
       int stage = 0;
       uint32_t phase = 0;
       int buf = 0;
@@ -254,7 +263,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const uint64_t da = smem_desc_sw128(sa + j * 32, 16, 1024);
             // B, MN-major: 64-column groups one TMA box (8 KiB) apart, 8-row k groups 1024 bytes
             // apart; 16 k rows = 2048 bytes.
-            const uint64_t db = smem_desc_sw128(sb + j * 2048, kBoxBytesB, 1024);
+            // (K-major B: like A -- its 64-row boxes follow each other, 8-row groups 1024 bytes
+            // apart, 32 bytes per K step.)
+            const uint64_t db = p.bt ? smem_desc_sw128(sb + j * 32, 16, 1024)
+                                     : smem_desc_sw128(sb + j * 2048, kBoxBytesB, 1024);
             if constexpr (kPair) mma_bf16_ss_pair(d_tmem, da, db, idesc, (kb | j) != 0 ? 1u : 0u);
             else mma_bf16_ss(d_tmem, da, db, idesc, (kb | j) != 0 ? 1u : 0u);
           }
@@ -391,6 +403,7 @@ constexpr int kSwapPrefetchBlocks = MORELLO_SWAP_PREFETCH_BLOCKS;   // k blocks 
 
 struct SwapParams {
   float* C;
+  int bt;           // 1: B is stored column-major, [b][n][k]
   int overwrite;    // 1: C = product instead of C += product
   int64_t m, n;
   int64_t c_batch;  // m * n
@@ -434,8 +447,13 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     tma_prefetch_descriptor(&map_b);
     const int ahead = min(p.k_blocks, kSwapPrefetchBlocks);
     for (int kb = 0; kb < ahead; ++kb) {
-      tma_prefetch_l2_3d(&map_b, col0, kb * kTileK, bb);
-      tma_prefetch_l2_3d(&map_b, col0 + 64, kb * kTileK, bb);
+      if (p.bt) {
+        tma_prefetch_l2_3d(&map_b, kb * kTileK, col0, bb);
+        tma_prefetch_l2_3d(&map_b, kb * kTileK, col0 + 64, bb);
+      } else {
+        tma_prefetch_l2_3d(&map_b, col0, kb * kTileK, bb);
+        tma_prefetch_l2_3d(&map_b, col0 + 64, kb * kTileK, bb);
+      }
     }
   }
   if (warp == 1) {
@@ -461,8 +479,13 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         uint8_t* sb = stages + (size_t)stage * S::kStageBytes;
         uint8_t* sa = sb + S::kBytesStrip;
         mbar_arrive_expect_tx(&bars->full[stage], S::kStageBytes);
-        tma_load_3d(sb, &map_b, &bars->full[stage], col0, kb * kTileK, bb);
-        tma_load_3d(sb + kBoxBytesB, &map_b, &bars->full[stage], col0 + 64, kb * kTileK, bb);
+        if (p.bt) {
+          tma_load_3d(sb, &map_b, &bars->full[stage], kb * kTileK, col0, bb);
+          tma_load_3d(sb + kBoxBytesB, &map_b, &bars->full[stage], kb * kTileK, col0 + 64, bb);
+        } else {
+          tma_load_3d(sb, &map_b, &bars->full[stage], col0, kb * kTileK, bb);
+          tma_load_3d(sb + kBoxBytesB, &map_b, &bars->full[stage], col0 + 64, kb * kTileK, bb);
+        }
         tma_load_3d(sa, &map_a, &bars->full[stage], kb * kTileK, 0, bb);
         if (++stage == S::kStages) { stage = 0; phase ^= 1; }
       }
@@ -473,7 +496,9 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     // ---------------------------------------------------------------- MMA issuer
     if (elect_one()) {
       // M = 128 columns of B (MN-major A operand), N = kRowsA rows of A (K-major B operand).
-      constexpr uint32_t idesc = instr_desc_bf16(kSwapStripCols, kRowsA, true, false);
+      // (With B column-major the strip is a K-major operand like the rows of A.)
+      const uint32_t idesc = p.bt ? instr_desc_bf16(kSwapStripCols, kRowsA, false, false)
+                                  : instr_desc_bf16(kSwapStripCols, kRowsA, true, false);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -487,7 +512,8 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           // The strip of B: 64-column groups one TMA box apart, 8-row k groups 1024 bytes
           // apart, 16 k rows = 2048 bytes.  The rows of A: 8-row groups 1024 bytes apart,
           // 16 k elements = 32 bytes along the row.
-          const uint64_t d_strip = smem_desc_sw128(sb + j * 2048, kBoxBytesB, 1024);
+          const uint64_t d_strip = p.bt ? smem_desc_sw128(sb + j * 32, 16, 1024)
+                                        : smem_desc_sw128(sb + j * 2048, kBoxBytesB, 1024);
           const uint64_t d_rows = smem_desc_sw128(sa + j * 32, 16, 1024);
           mma_bf16_ss(tmem_base, d_strip, d_rows, idesc, (kb | j) != 0 ? 1u : 0u);
         }
@@ -540,8 +566,10 @@ struct MapKey {
   const void* b;
   const void* c;
   int64_t bsz, m, k, n;
+  bool bt;   // B column-major
   bool operator==(const MapKey& o) const {
-    return a == o.a && b == o.b && c == o.c && bsz == o.bsz && m == o.m && k == o.k && n == o.n;
+    return a == o.a && b == o.b && c == o.c && bsz == o.bsz && m == o.m && k == o.k && n == o.n &&
+           bt == o.bt;
   }
 };
 struct MapEntry {
@@ -576,9 +604,16 @@ cudaError_t get_maps(const MapKey& key, CUtensorMap* ma, CUtensorMap* mb, CUtens
                                        (uint64_t)key.k, (uint64_t)key.m, (uint64_t)key.bsz, kTileK,
                                        (uint32_t)a_box_rows(key.m), CU_TENSOR_MAP_SWIZZLE_128B);
   if (err != cudaSuccess) return err;
-  err = make_tensor_map_3d(&e.map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, key.b, (uint64_t)key.n,
-                           (uint64_t)key.k, (uint64_t)key.bsz, 64, kTileK,
-                           CU_TENSOR_MAP_SWIZZLE_128B);
+  // Either way a box is 64 x 64 elements with 128-byte rows: [k][n] gives 64 k rows of 64
+  // columns, [n][k] gives 64 columns (rows of the stored matrix) of 64 k.
+  if (key.bt)
+    err = make_tensor_map_3d(&e.map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, key.b, (uint64_t)key.k,
+                             (uint64_t)key.n, (uint64_t)key.bsz, kTileK, 64,
+                             CU_TENSOR_MAP_SWIZZLE_128B);
+  else
+    err = make_tensor_map_3d(&e.map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, key.b, (uint64_t)key.n,
+                             (uint64_t)key.k, (uint64_t)key.bsz, 64, kTileK,
+                             CU_TENSOR_MAP_SWIZZLE_128B);
   if (err != cudaSuccess) return err;
   err = make_tensor_map_3d(&e.map_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, key.c, (uint64_t)key.n,
                            (uint64_t)key.m, (uint64_t)key.bsz, kEpiCols, 32,
@@ -721,7 +756,7 @@ namespace {
 template <bool kPair, int kTileN>
 cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, int64_t n,
                         const CUtensorMap& map_a, const CUtensorMap& map_b,
-                        const CUtensorMap& map_c, float* C, bool halves, bool overwrite,
+                        const CUtensorMap& map_c, float* C, bool halves, bool overwrite, bool bt,
                         cudaStream_t stream) {
   using S = Shape<kPair, kTileN>;
   const cudaError_t attr_err = set_smem_attribute<kPair, kTileN>();
@@ -740,6 +775,7 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   p.status = dev.status;
   p.a_box_rows = a_box_rows(m);
   p.overwrite = overwrite ? 1 : 0;
+  p.bt = bt ? 1 : 0;
 
   const int64_t max_units = kPair ? pair_units(dev.sms) : dev.sms;
   // The last wave of a compute-bound problem: when its tiles would occupy at most half the
@@ -779,7 +815,7 @@ namespace {
 template <int kRowsA>
 cudaError_t launch_swap(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, int64_t n,
                         const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
-                        bool overwrite, cudaStream_t stream, uint64_t* launches) {
+                        bool overwrite, bool bt, cudaStream_t stream, uint64_t* launches) {
   using S = SwapShape<kRowsA>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
@@ -789,6 +825,7 @@ cudaError_t launch_swap(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   });
   if (attr_err != cudaSuccess) return attr_err;
   SwapParams p{};
+  p.bt = bt ? 1 : 0;
   p.overwrite = overwrite ? 1 : 0;
   p.m = m; p.n = n;
   p.c_batch = m * n;
@@ -820,21 +857,21 @@ cudaError_t launch_swap(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
 
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m, int64_t k,
                         int64_t n, const uint16_t* A, const uint16_t* B, float* C, float*,
-                        cudaStream_t stream, uint64_t* launches, bool overwrite) {
+                        cudaStream_t stream, uint64_t* launches, bool overwrite, bool bt) {
   CUtensorMap map_a, map_b, map_c;
-  cudaError_t e = get_maps(MapKey{A, B, C, b, m, k, n}, &map_a, &map_b, &map_c);
+  cudaError_t e = get_maps(MapKey{A, B, C, b, m, k, n, bt}, &map_a, &map_b, &map_c);
   if (e != cudaSuccess) return e;
   const int code = plan.form * 1000 + plan.tile_n;
   switch (code) {
-    case 3016: return launch_swap<16>(dev, b, m, k, n, map_a, map_b, C, overwrite, stream, launches);
-    case 3032: return launch_swap<32>(dev, b, m, k, n, map_a, map_b, C, overwrite, stream, launches);
-    case 3048: return launch_swap<48>(dev, b, m, k, n, map_a, map_b, C, overwrite, stream, launches);
-    case 3064: return launch_swap<64>(dev, b, m, k, n, map_a, map_b, C, overwrite, stream, launches);
-    case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, stream); break;
-    case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, stream); break;
-    case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, stream); break;
-    case 2128: e = launch_gemm<true, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, stream); break;
-    case 2256: e = launch_gemm<true, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, stream); break;
+    case 3016: return launch_swap<16>(dev, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
+    case 3032: return launch_swap<32>(dev, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
+    case 3048: return launch_swap<48>(dev, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
+    case 3064: return launch_swap<64>(dev, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
+    case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, bt, stream); break;
+    case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, bt, stream); break;
+    case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, bt, stream); break;
+    case 2128: e = launch_gemm<true, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, bt, stream); break;
+    case 2256: e = launch_gemm<true, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, bt, stream); break;
     default: return cudaErrorInvalidValue;
   }
   if (e == cudaSuccess) ++*launches;

@@ -97,6 +97,13 @@ int gemm_pair_units(int sms);
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m,
                         int64_t k, int64_t n, const uint16_t* A, const uint16_t* B, float* C,
                         float* workspace, cudaStream_t stream, uint64_t* launches,
-                        bool overwrite = false);
+                        bool overwrite = false, bool b_col_major = false);
+
+// ---- B stored column-major where the TMA engine cannot address it ------------
+// C[b, i, j] (+)= sum_p A[b, i, p] * Bt[b, j, p]: one warp per output column, lanes stride over
+// k, shuffle sums in a fixed order.  Any shape, no alignment needs; slow, deterministic.
+cudaError_t colmajor_fallback_launch(int64_t b, int64_t m, int64_t k, int64_t n, const uint16_t* A,
+                                     const uint16_t* Bt, float* C, bool overwrite,
+                                     cudaStream_t stream, uint64_t* launches);
 
 }  // namespace morello

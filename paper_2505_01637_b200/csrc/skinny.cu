@@ -387,6 +387,49 @@ cudaError_t skinny_launch(const SkinnyPlan& plan, int64_t b, int m, int64_t k, i
   return cudaSuccess;
 }
 
+namespace {
+
+// One warp per output column j of one batch: lane l visits k = l, l + 32, ... of row j of Bt
+// (coalesced) for every row i of A in turn.
+__global__ void __launch_bounds__(256)
+colmajor_fallback_kernel(const uint16_t* __restrict__ A, const uint16_t* __restrict__ Bt,
+                         float* __restrict__ C, int64_t m, int64_t k, int64_t n, int overwrite) {
+  const int lane = threadIdx.x & 31;
+  const int64_t j = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int64_t bb = blockIdx.y;
+  if (j >= n) return;
+  const uint16_t* brow = Bt + (bb * n + j) * k;
+  for (int64_t i = 0; i < m; ++i) {
+    const uint16_t* arow = A + (bb * m + i) * k;
+    float sum = 0.f;
+    for (int64_t p = lane; p < k; p += 32)
+      sum = fmaf(__uint_as_float(((uint32_t)arow[p]) << 16), __uint_as_float(((uint32_t)brow[p]) << 16), sum);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    if (lane == 0) {
+      float* c = C + (bb * m + i) * n + j;
+      *c = overwrite ? sum : *c + sum;
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t colmajor_fallback_launch(int64_t b, int64_t m, int64_t k, int64_t n, const uint16_t* A,
+                                     const uint16_t* Bt, float* C, bool overwrite,
+                                     cudaStream_t stream, uint64_t* launches) {
+  for (int64_t b0 = 0; b0 < b; b0 += 65535) {
+    const int64_t bn = std::min<int64_t>(65535, b - b0);
+    dim3 grid((unsigned)((n + 7) / 8), (unsigned)bn, 1);
+    colmajor_fallback_kernel<<<grid, 256, 0, stream>>>(A + b0 * m * k, Bt + b0 * n * k, C + b0 * m * n,
+                                                       m, k, n, overwrite ? 1 : 0);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    ++*launches;
+  }
+  return cudaSuccess;
+}
+
 cudaError_t skinny_reduce_launch(const float* partial, float* C, int64_t b, int m, int64_t n,
                                  int64_t c_batch, int split_k, cudaStream_t stream, bool overwrite) {
   const int64_t total = b * m * n;

@@ -387,3 +387,26 @@ def test_f32_oracle_one_hot_layout_abs_dot_and_float64_agreement():
     ref = C.astype(np.float64) + np.einsum("bik,bkj->bij", A.astype(np.float64), B.astype(np.float64))
     assert np.abs(got - ref).max() <= np.spacing(np.abs(ref).max().astype(np.float32))
     assert np.allclose(T, np.einsum("bik,bkj->bij", np.abs(A).astype(np.float64), np.abs(B).astype(np.float64)), rtol=1e-12)
+
+
+# ------------------------------------------------ column-major right-hand side (Section 2.2's
+# Spec example has a col_major rhs): pinned to the row-major oracle and to a one-hot
+def test_colmajor_oracle_equals_rowmajor_oracle_on_the_transposed_operand():
+    for (b, m, k, n) in [(1, 4, 128, 16), (2, 3, 65, 40), (3, 1, 7, 9)]:      # first: the Spec example's shape
+        A, B, C = w.make(b, m, k, n, seed=21 + k, ab="uniform", c="normal")
+        Bt = np.ascontiguousarray(B.transpose(0, 2, 1))
+        assert np.array_equal(bits(oracle.matmul_accum_bt(b, m, k, n, A, Bt, C)),
+                              bits(oracle.matmul_accum(b, m, k, n, A, B, C)))
+
+
+def test_colmajor_oracle_one_hot_pins_the_indexing():
+    b, m, k, n = 2, 3, 5, 4
+    rng = np.random.default_rng(9)
+    Av = rng.integers(-100, 101, size=(b, m, k)).astype(np.float32)
+    C = rng.integers(-50, 51, size=(b, m, n)).astype(np.float32)
+    Bt1 = np.zeros((b, n, k), np.float32)
+    Bt1[1, 2, 3] = -3.0                                  # B[1][p=3][j=2]
+    want = C.copy()
+    want[1, :, 2] += -3.0 * Av[1, :, 3]
+    got = oracle.matmul_accum_bt(b, m, k, n, as_bf16(Av), as_bf16(Bt1), C)
+    assert np.array_equal(got, want)
