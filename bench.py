@@ -461,6 +461,16 @@ def run_ours(args):
         raise RuntimeError("device status %d (0x%x)" % (st, detail))
     value = whole_job_value(cfg.algorithmic_bytes, args.steps, world, sec) / 1e9
 
+    # ---- the same calls on ONE set of buffers (how the config is worded: "timed warm over 1000
+    # calls"); B's 64 MiB fit the 126 MB L2, so this figure is L2-assisted and is not the headline
+    def step_same(i):
+        rc = call(b, m, k, n, pa, pbs[0], pcs[0], stream)
+        if rc != 0:
+            raise mb.MorelloError(rc, "bench step")
+    t0 = time.perf_counter()
+    same_us = time_calls(torch, step_same, args.steps, args.warmup) / args.steps * 1e6
+    windows.append((t0, time.perf_counter()))
+
     # ---- the same loop replayed from a CUDA graph (launch overhead taken out)
     graph_us = None
     try:
@@ -564,6 +574,9 @@ def run_ours(args):
                          "peak_kind": peak_kind, "frac_of_nominal_8TBs": per_launch_gbs / NOMINAL_HBM_GBS,
                          "traffic": traffic.get(cfg.name), "kernel": "gemv_stream_kernel<1>"},
             "graph_replay_us_per_call": graph_us,
+            "same_buffer_us_per_call": same_us,
+            "same_buffer_note": "one B buffer re-read every call: 64 MiB < L2, L2-assisted, not an HBM figure",
+            "inputs_crc32": {"A": w.crc32(A), "B0": w.crc32(B0), "C": w.crc32(C)},
             "cpu_baseline": cpu,
             "configs": extra,
         }

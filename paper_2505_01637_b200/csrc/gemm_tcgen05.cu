@@ -832,24 +832,23 @@ cudaError_t launch_swap(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   p.k_blocks = (int)((k + kTileK - 1) / kTileK);
   p.status = dev.status;
   const int64_t strips = (n + kSwapStripCols - 1) / kSwapStripCols;
-  // grid.y carries the batch index (the tensor maps cover all batches); larger batches in slabs
-  for (int64_t b0 = 0; b0 < b; b0 += 65535) {
-    if (b0 != 0) return cudaErrorInvalidValue;   // the planner keeps such batches off this form
-    p.C = C;
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3((unsigned)strips, (unsigned)std::min<int64_t>(b, 65535), 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = S::kSmemBytes;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, swap_kernel<kRowsA>, map_a, map_b, p);
-    if (e != cudaSuccess) return e;
-    ++*launches;
-  }
+  // grid.y carries the batch index (the planner keeps batches beyond a grid dimension off
+  // this kernel).
+  if (b > 65535) return cudaErrorInvalidValue;
+  p.C = C;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)strips, (unsigned)b, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = S::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, swap_kernel<kRowsA>, map_a, map_b, p);
+  if (e != cudaSuccess) return e;
+  ++*launches;
   return cudaSuccess;
 }
 
