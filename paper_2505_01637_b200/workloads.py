@@ -125,7 +125,7 @@ def make(b, m, k, n, seed, ab="uniform", c="normal"):
 
 
 def make_config(index: int, variant: str = "random"):
-    """Inputs of BASELINE config ``index`` (0-based).
+    """Inputs of benchmark configuration ``index`` (0-based).
 
     variant: "random" (the config's own distributions), "integer" (A, B integer
     uniform in [-4, 4], C as the config says) or "integer_intc" (C integers in
