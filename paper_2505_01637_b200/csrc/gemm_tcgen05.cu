@@ -375,13 +375,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 // follows m instead of a fixed 128 rows, the accumulator is 128 lanes x kRowsA columns, and
 // the epilogue holds one column of C per thread: for every row i a warp adds 32 consecutive
 // floats of C (C is read before the main loop, the sum is added once, at the end).
-// The call streams B once and is bound by HBM, so the block is kept small enough (at most
-// 108 KiB of stages, 32 or 64 TMEM columns) for the next call's block to be resident beside
-// it: before its griddepcontrol.wait that block asks the TMA engine to prefetch its first k
+// The call streams B once and is bound by HBM.  Up to 16 rows the block is kept small enough
+// (108 KiB of stages, 32 TMEM columns) for the next call's block to be resident beside it:
+// before its griddepcontrol.wait that block asks the TMA engine to prefetch its first k
 // blocks of B into L2 (nothing reaches the SM, so this is legal early), and a block lets
-// dependents launch once its producer has issued its last load.
+// dependents launch once its producer has issued its last load.  With more rows a stage
+// carries more of A and the same budget would hold too little of B in flight: the ring then
+// takes 200 KiB and the next call's block follows when this one leaves (measured, 2048 x
+// 16384, 108 / 200 KiB: 32 rows 12.9 / 12.6 us, 48 rows 14.8 / 13.1, 64 rows 15.4 / 13.8).
 #ifndef MORELLO_SWAP_RING_KIB
-#define MORELLO_SWAP_RING_KIB 108        // shared memory for the stages: two blocks fit an SM
+#define MORELLO_SWAP_RING_KIB 108        // stages of the <= 16-row kernel: two blocks fit an SM
+#endif
+#ifndef MORELLO_SWAP_BIG_RING_KIB
+#define MORELLO_SWAP_BIG_RING_KIB 200    // stages with more rows of A
 #endif
 #ifndef MORELLO_SWAP_PREFETCH_BLOCKS
 #define MORELLO_SWAP_PREFETCH_BLOCKS 6
@@ -391,14 +397,15 @@ struct SwapShape {
   static constexpr int kBytesStrip = 2 * kBoxBytesB;                  // 128 columns x 64 k: 16 KiB
   static constexpr int kBytesRows = kRowsA * kTileK * 2;              // 2 .. 8 KiB
   static constexpr int kStageBytes = kBytesStrip + kBytesRows;
-  static constexpr int kFit = (MORELLO_SWAP_RING_KIB * 1024) / kStageBytes;
+  static constexpr int kRingKiB = kRowsA <= 16 ? MORELLO_SWAP_RING_KIB : MORELLO_SWAP_BIG_RING_KIB;
+  static constexpr int kFit = (kRingKiB * 1024) / kStageBytes;
   static constexpr int kStages = kFit < kMaxStages ? kFit : kMaxStages;
   static constexpr int kTmemCols = kRowsA <= 32 ? 32 : 64;
   static constexpr size_t kSmemBytes = (size_t)kStages * kStageBytes + 1024 /*alignment slack*/ + 256;
   static_assert(kRowsA % 16 == 0 && kRowsA >= 16 && kRowsA <= 64, "rows of A");
 };
 constexpr int kSwapStripCols = 128;
-constexpr int kSwapAutoRows = 32;        // the planner picks this kernel up to this many rows
+constexpr int kSwapMaxRows = 64;
 constexpr int kSwapPrefetchBlocks = MORELLO_SWAP_PREFETCH_BLOCKS;   // k blocks asked into L2 before the wait
 
 struct SwapParams {
@@ -708,13 +715,15 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t, int64_t n, int knob) 
   const bool halves = (knob / 256) == 0;
   knob %= 256;
   int form = knob % 16, tile_n = (knob / 16) * 64;
-  // Form 3: the operand-swapped kernel for few rows.  By shape it takes every call of at most
-  // 32 rows whose strips of 128 columns occupy at least half the SMs (measured on 2048 x 16384,
-  // us per call, swapped / 128-row tiles: m = 16: 11.7 / 14.2, 32: 12.7 / 14.4, 48: 14.6 / 14.6,
-  // 64: 15.5 / 14.8 -- with more rows of A per stage the ring gets shallower).
-  if (form == 3 || (form == 0 && tile_n == 0 && m <= kSwapAutoRows && b <= 65535 &&
+  // Form 3: the operand-swapped kernel.  By shape it takes every call of at most 64 rows whose
+  // strips of 128 columns occupy at least half the SMs (measured on 2048 x 16384, us per call,
+  // swapped / 128-row tiles: m = 16: 11.7 / 14.2, 32: 12.6 / 14.4, 48: 13.1 / 14.6, 64: 13.8 / 14.9).
+  // Beyond 64 rows the 128-row tiles win: an accumulator of more than 64 columns per thread
+  // cannot be paired with an early read of C in registers, and sending the sums out as L2
+  // reductions instead cost more than it saved (96 rows: 16.7 against 15.4 us).
+  if (form == 3 || (form == 0 && tile_n == 0 && m <= kSwapMaxRows && b <= 65535 &&
                     b * ((n + kSwapStripCols - 1) / kSwapStripCols) * 2 >= sms)) {
-    if (m > 64 || tile_n != 0 || b > 65535) return GemmPlan{false, 0, 0, 0, false};
+    if (m > kSwapMaxRows || tile_n != 0 || b > 65535) return GemmPlan{false, 0, 0, 0, false};
     return GemmPlan{true, 3, a_box_rows(m), 0, false};
   }
   if (form < 0 || form > 2 || (tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) ||

@@ -135,6 +135,7 @@ SWAP = 3
     (1, 33, 264, 520),      # 48-row instantiation
     (1, 49, 128, 392),      # 64-row instantiation
     (1, 64, 2048, 1024),
+    (2, 60, 136, 264),
     (1, 16, 2048, 16384),   # the decode-style config
 ])
 def test_swap_form_matches_oracle(shape):
