@@ -73,9 +73,9 @@ int morello_matmul_accum(int64_t b, int64_t m, int64_t k, int64_t n,
                          const void* A, const void* B, float* C, void* stream);
 
 /*
- * Bytes of scratch morello_matmul_accum_ws needs for this shape on the current
- * device (0 if none; also 0 for invalid shapes).  The figure assumes A, B and
- * C are 16-byte aligned; it is an upper bound otherwise.
+ * Bytes of scratch that suffice for morello_matmul_accum_ws on this shape on the
+ * current device, whatever the alignment of A, B and C turns out to be (the kernel
+ * chosen depends on it): 0 if none can be needed; also 0 for invalid shapes.
  */
 size_t morello_workspace_bytes(int64_t b, int64_t m, int64_t k, int64_t n);
 

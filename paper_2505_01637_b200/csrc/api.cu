@@ -277,7 +277,13 @@ int morello_matmul_accum(int64_t b, int64_t m, int64_t k, int64_t n, const void*
 }
 
 size_t morello_workspace_bytes(int64_t b, int64_t m, int64_t k, int64_t n) {
-  return morello_workspace_bytes_forced(MORELLO_PATH_AUTO, 0, b, m, k, n);
+  // The selector looks at the pointers' alignment too, which is not known here: operands that
+  // are not 16-byte aligned turn a tensor-core call into an FMA call, whose k slices need
+  // scratch.  The answer covers every path the call could take.
+  const size_t chosen = morello_workspace_bytes_forced(MORELLO_PATH_AUTO, 0, b, m, k, n);
+  const size_t fma_register = morello_workspace_bytes_forced(MORELLO_PATH_SKINNY, kKnobSplitMod * SKINNY_REGISTER, b, m, k, n);
+  const size_t fma_any = morello_workspace_bytes_forced(MORELLO_PATH_SKINNY, 0, b, m, k, n);
+  return std::max(chosen, std::max(fma_register, fma_any));
 }
 
 size_t morello_workspace_bytes_forced(int path, int split_k, int64_t b, int64_t m, int64_t k,

@@ -39,7 +39,6 @@ struct SkinnyParams {
   int col_blocks;
   int split_k;
   int k_chunk;
-  int early_b;  // 1: B may be fetched before the preceding kernel on the stream has completed
   int overwrite;  // 1: C = sum instead of C += sum
 };
 
@@ -148,14 +147,11 @@ skinny_kernel(const SkinnyParams p) {
   const uint16_t* a_base = p.A + (int64_t)bb * p.a_batch;
   const uint16_t* bp = p.B + (int64_t)bb * p.b_batch + (int64_t)unit * VEC + (k0 + rl) * p.n;
 
-  // The first group of B rows is requested before A is staged, so that the
-  // staging latency hides under the first HBM round trip.  When the caller has
-  // declared B stable (early_b), it is requested even before the preceding
-  // kernel on the stream is known to have completed; A, C and the partial sums
-  // are only touched after pdl_wait().
+  // The first group of B rows is requested before A is staged, so that the staging
+  // latency hides under the first HBM round trip.  Nothing is touched before pdl_wait().
   BVec<VEC> v[UNROLL];
   bool preloaded = false;
-  if (p.early_b) pdl_release(); else pdl_wait();
+  pdl_wait();
   if (active) {
     const int kcl0 = (int)min((int64_t)p.k_chunk, k1 - k0);
 #pragma unroll
@@ -163,7 +159,7 @@ skinny_kernel(const SkinnyParams p) {
       if (rl + u * R < kcl0) v[u].load(bp + u * step);
     preloaded = true;
   }
-  if (p.early_b) pdl_wait(); else pdl_release();
+  pdl_release();
 
   for (int64_t kc0 = k0; kc0 < k1; kc0 += p.k_chunk) {
     const int kcl = (int)min((int64_t)p.k_chunk, k1 - kc0);

@@ -47,3 +47,22 @@ def test_misaligned_a_or_c_take_the_fma_kernels_with_the_same_result():
     torch.cuda.synchronize()
     assert_bit_exact(bigC[1:1 + C.size].cpu().numpy().reshape(b, m, n), want, "C misaligned for TMA")
     assert float(bigC[0]) == 0.0
+
+
+def test_workspace_query_covers_the_path_a_misaligned_operand_falls_to():
+    b, m, k, n = 1, 40, 8192, 64         # aligned: tensor-core tiles, no scratch; A off by 2 bytes: FMA kernel, k in slices
+    A, B, C = w.make(b, m, k, n, seed=6, ab="int4", c="int8")
+    want = oracle.matmul_accum(b, m, k, n, A, B, C)
+    need = mb.morello_workspace_bytes(b, m, k, n)
+    assert need > 0
+    dA, dB, dC = to_dev(A, B, C)
+    bigA = torch.zeros(A.size + 8, dtype=torch.int16, device="cuda")
+    bigA[1:1 + A.size] = dA.reshape(-1)
+    ws = torch.empty(need // 4 + 4, device="cuda")
+    mb.morello_matmul_accum_ws(b, m, k, n, bigA[1:], dB, dC, ws, need)
+    torch.cuda.synchronize()
+    assert_bit_exact(dC.cpu().numpy(), want, "_ws with a misaligned A")
+    dC2 = torch.from_numpy(C.copy()).cuda()
+    mb.morello_matmul_accum_ws(b, m, k, n, dA, dB, dC2, ws, need)      # aligned: same buffer suffices
+    torch.cuda.synchronize()
+    assert_bit_exact(dC2.cpu().numpy(), want, "_ws with aligned operands")
