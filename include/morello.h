@@ -200,7 +200,9 @@ int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n);
  * that split and (value / 1024) picks the kernel: 0 = by shape, 1 = the register-
  * streaming kernel (any shape), 2 = the TMA-ring GEMV kernel (m <= 4, n % 8 == 0,
  * 16-byte-aligned B; it raises the split as needed to keep the part of A a block
- * stages within 32 KiB: 16384 / m rows of k per block, m rounded up to 1, 2 or 4).  On the tcgen05 path, which never
+ * stages within 32 KiB: 16384 / m rows of k per block, m rounded up to 1, 2 or 4; up to
+ * 8 slices are added inside a thread-block cluster, without scratch), 3 = the same kernel
+ * with the slices always added by the reduce kernel from scratch.  On the tcgen05 path, which never
  * splits k, the argument instead selects the tile: (value % 16) is the form -- 0 = by
  * shape, 1 = one CTA per 128-row tile, 2 = a pair of CTAs per 256-row tile
  * (cta_group::2), 3 = the operand-swapped kernel for at most 64 rows (no column count

@@ -109,9 +109,11 @@ int select_path(int sms, int64_t b, int64_t m, int64_t k, int64_t n, const void*
 // The knob of the forced entry point on the skinny path: knob % 1024 is the split of the k
 // range (0 = automatic), knob / 1024 picks the kernel (0 = by shape, 1 = the register-
 // streaming kernel, 2 = the TMA-ring GEMV kernel, which needs m <= 4, n % 8 == 0 and a
-// 16-byte-aligned B).
+// 16-byte-aligned B, 3 = the same with the k slices always added by the reduce kernel from
+// scratch instead of inside a cluster).
 constexpr int kKnobSplitMod = 1024;
-enum { SKINNY_AUTO = 0, SKINNY_REGISTER = 1, SKINNY_STREAM = 2 };
+enum { SKINNY_AUTO = 0, SKINNY_REGISTER = 1, SKINNY_STREAM = 2, SKINNY_STREAM_SCRATCH = 3 };
+inline bool knob_scratch_reduce(int knob) { return knob / kKnobSplitMod == SKINNY_STREAM_SCRATCH; }
 
 // Which skinny kernel runs this shape: -1 = the request cannot be met.
 int skinny_kernel_for(int knob, int64_t b, int64_t m, int64_t k, int64_t n, const void* B) {
@@ -119,7 +121,7 @@ int skinny_kernel_for(int knob, int64_t b, int64_t m, int64_t k, int64_t n, cons
   const bool can = m <= 4 && stream_shape_supported(b, (int)m, k, n, B) &&
                    stream_plan(1, b, (int)m, k, n, knob % kKnobSplitMod).supported;
   if (want == SKINNY_REGISTER) return SKINNY_REGISTER;
-  if (want == SKINNY_STREAM) return can ? SKINNY_STREAM : -1;
+  if (want == SKINNY_STREAM || want == SKINNY_STREAM_SCRATCH) return can ? SKINNY_STREAM : -1;
   if (want != SKINNY_AUTO) return -1;
   // Small problems finish inside one launch latency either way; the ring pays off once
   // there is a stream of B worth pipelining.
@@ -131,7 +133,8 @@ int skinny_kernel_for(int knob, int64_t b, int64_t m, int64_t k, int64_t n, cons
 size_t skinny_workspace(int sms, int64_t b, int64_t m, int64_t k, int64_t n, const void* B, int knob) {
   const int split_k = knob % kKnobSplitMod;
   const int which = skinny_kernel_for(knob, b, m, k, n, B);
-  if (which == SKINNY_STREAM) return stream_plan(sms, b, (int)m, k, n, split_k).workspace_bytes;
+  if (which == SKINNY_STREAM)
+    return stream_plan(sms, b, (int)m, k, n, split_k, knob_scratch_reduce(knob)).workspace_bytes;
   const int vec = skinny_vec(n, B);
   // Chunks are full (16 rows) except possibly the last one.
   const int first = (int)std::min<int64_t>(kSkinnyMaxRows, m);
@@ -245,7 +248,8 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     e = gemm_launch(st->info, plan, b, m, k, n, static_cast<const uint16_t*>(A),
                     static_cast<const uint16_t*>(B), C, ws, s, &launches, overwrite);
   } else if (which == SKINNY_STREAM) {
-    const StreamPlan plan = stream_plan(sms, b, (int)m, k, n, split_k % kKnobSplitMod);
+    const StreamPlan plan = stream_plan(sms, b, (int)m, k, n, split_k % kKnobSplitMod,
+                                        knob_scratch_reduce(split_k));
     e = stream_launch(st->info, plan, b, (int)m, k, n, static_cast<const uint16_t*>(A), m * k,
                       static_cast<const uint16_t*>(B), C, m * n, ws, s, &launches, overwrite);
   } else {

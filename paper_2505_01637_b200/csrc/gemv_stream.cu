@@ -14,8 +14,11 @@
 //               then frees the stage on its "empty" mbarrier.
 // At the end the four row groups of a warp are added with shuffles and the eight warps
 // through shared memory, always in the same order, so results are deterministic.  With one
-// slice the block adds its sums to C (C was read early, the addition happens once, last);
-// with several it writes partial[slice][b][m][n] for the slice-ordered reduce kernel.
+// slice the block adds its sums to C (C was read early, the addition happens once, last).
+// With 2, 4 or 8 slices the blocks of a strip form a thread-block cluster: each parks its
+// sums in its own shared memory and block 0 reads them through distributed shared memory in
+// slice order, adds C and stores -- one launch, no scratch, a fixed order.  More slices (a
+// forced split) write partial[slice][b][m][n] for the slice-ordered reduce kernel.
 //
 // Between back-to-back calls.  The kernel is launched with programmatic stream
 // serialisation.  Before griddepcontrol.wait it only sets up barriers and asks the TMA
@@ -66,6 +69,7 @@ constexpr int kConsumers = 32 * kConsumerWarps;
 constexpr int kThreads = 32 + kConsumers;
 constexpr int kMaxSliceBytes = 32 * 1024;                   // bf16 rows of A staged per block
 constexpr int max_slice_k(int m_tile) { return kMaxSliceBytes / (2 * m_tile); }
+constexpr int kMaxClusterK = 8;                             // k slices added inside one cluster
 constexpr int kPrefetchBoxes = MORELLO_GEMV_PREFETCH_BOXES; // boxes asked into L2 before the wait
 constexpr int kLanesPerRow = kStripCols / 8;                // 16-byte chunks per box row
 constexpr int kRowsPerWarp = 32 / kLanesPerRow;             // box rows one warp-wide load covers
@@ -85,6 +89,8 @@ struct StreamParams {
   int split_k;
   int k_per_split;                // multiple of kBoxRows
   int overwrite;                  // 1: C = sum instead of C += sum
+  int cluster_k;                  // 1: the k slices of a strip form a thread-block cluster and are
+                                  //    added through distributed shared memory (no scratch)
   int a_bulk;                     // rows of A can be brought by bulk copies (16-byte alignment)
   uint32_t* status;
 };
@@ -122,7 +128,7 @@ __device__ __forceinline__ void fma2(uint64_t& acc, uint64_t a, uint64_t b) {
 #endif
 }
 
-template <int M_T>
+template <int M_T, bool kClusterK>
 __global__ void __launch_bounds__(kThreads)
 gemv_stream_kernel(const __grid_constant__ CUtensorMap map_b, const StreamParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -130,13 +136,16 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_b, const StreamParams
       (reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
   uint16_t* a_s = reinterpret_cast<uint16_t*>(ring + kStages * kStageBytes);  // [M_T][k_per_split] bf16
   float* red = reinterpret_cast<float*>(a_s + (size_t)p.k_per_split * M_T);   // [warp][M_T][64]
-  StreamBarriers* bars = reinterpret_cast<StreamBarriers*>(red + kConsumerWarps * M_T * kStripCols);
+  float* out_s = red + kConsumerWarps * M_T * kStripCols;                     // [M_T][64]: this block's sums
+  StreamBarriers* bars = reinterpret_cast<StreamBarriers*>(out_s + M_T * kStripCols);
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int strip = blockIdx.x % p.strips;
-  const int slice = blockIdx.x / p.strips;
+  // Cluster form: the split_k blocks of a strip are consecutive (they are one cluster and the
+  // slice is the block's rank in it); otherwise slices are the slow index.
+  const int strip = kClusterK ? blockIdx.x / p.split_k : blockIdx.x % p.strips;
+  const int slice = kClusterK ? blockIdx.x % p.split_k : blockIdx.x / p.strips;
   const int bb = blockIdx.y;
   const int k0 = slice * p.k_per_split;
   const int k1 = (int)min((int64_t)k0 + p.k_per_split, p.k);
@@ -221,7 +230,8 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_b, const StreamParams
     const int i = o / kStripCols;
     const int64_t col = col0 + (o % kStripCols);
     c_in[r] = 0.f;
-    if (p.split_k == 1 && !p.overwrite && o < M_T * kStripCols && i < p.m && col < p.n)
+    if ((p.split_k == 1 || (kClusterK && slice == 0)) && !p.overwrite && o < M_T * kStripCols &&
+        i < p.m && col < p.n)
       c_in[r] = p.C[(int64_t)bb * p.c_batch + (int64_t)i * p.n + col];
   }
   consumer_sync();
@@ -300,21 +310,53 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_b, const StreamParams
     }
   }
   consumer_sync();                        // reached by every consumer, timed out or not
-  if (*abort_flag) return;
+  if (!kClusterK && *abort_flag) return;
+  float sums[kOutPerThread];
 #pragma unroll
   for (int r = 0; r < kOutPerThread; ++r) {
     const int o = ct + r * kConsumers;
+    sums[r] = 0.f;
+    if (o >= M_T * kStripCols) continue;
     const int i = o / kStripCols;
-    const int64_t col = col0 + (o % kStripCols);
-    if (o >= M_T * kStripCols || i >= p.m || col >= p.n) continue;
     float sum = red[(size_t)i * kStripCols + (o % kStripCols)];
 #pragma unroll
     for (int w = 1; w < kConsumerWarps; ++w)
       sum += red[((size_t)w * M_T + i) * kStripCols + (o % kStripCols)];
-    if (p.split_k == 1)
-      p.C[(int64_t)bb * p.c_batch + (int64_t)i * p.n + col] = c_in[r] + sum;
-    else
-      p.partial[(int64_t)slice * p.partial_split_stride + ((int64_t)bb * p.m + i) * p.n + col] = sum;
+    sums[r] = sum;
+    if constexpr (kClusterK) out_s[o] = sum;
+  }
+  if constexpr (kClusterK) {
+    // Every block of the cluster has parked its sums; block 0 adds them in slice order
+    // (its own first), adds C once and stores.  The second barrier keeps the other blocks'
+    // shared memory alive until block 0 has read it.  Both barriers are reached by every
+    // consumer of every block, timed out or not (the producer warps have exited and do not
+    // count), so no block can be left waiting.
+    cluster_sync();
+    if (slice == 0 && !*abort_flag) {
+#pragma unroll
+      for (int r = 0; r < kOutPerThread; ++r) {
+        const int o = ct + r * kConsumers;
+        const int i = o / kStripCols;
+        const int64_t col = col0 + (o % kStripCols);
+        if (o >= M_T * kStripCols || i >= p.m || col >= p.n) continue;
+        float sum = sums[r];
+        for (int s2 = 1; s2 < p.split_k; ++s2) sum += ld_shared_cluster_f32(map_to_cta(smem_u32(out_s + o), s2));
+        p.C[(int64_t)bb * p.c_batch + (int64_t)i * p.n + col] = c_in[r] + sum;
+      }
+    }
+    cluster_sync();
+  } else {
+#pragma unroll
+    for (int r = 0; r < kOutPerThread; ++r) {
+      const int o = ct + r * kConsumers;
+      const int i = o / kStripCols;
+      const int64_t col = col0 + (o % kStripCols);
+      if (o >= M_T * kStripCols || i >= p.m || col >= p.n) continue;
+      if (p.split_k == 1)
+        p.C[(int64_t)bb * p.c_batch + (int64_t)i * p.n + col] = c_in[r] + sums[r];
+      else
+        p.partial[(int64_t)slice * p.partial_split_stride + ((int64_t)bb * p.m + i) * p.n + col] = sums[r];
+    }
   }
 }
 
@@ -367,13 +409,13 @@ cudaError_t get_b_map(const BKey& key, CUtensorMap* out) {
 
 size_t smem_for(int m_tile, int k_per_split) {
   return 128 + (size_t)kStages * kStageBytes + (size_t)k_per_split * m_tile * 2 +
-         (size_t)kConsumerWarps * m_tile * kStripCols * 4 + sizeof(StreamBarriers) + 16;
+         (size_t)(kConsumerWarps + 1) * m_tile * kStripCols * 4 + sizeof(StreamBarriers) + 16;
 }
 
-template <int M_T>
+template <int M_T, bool kClusterK>
 cudaError_t launch(const StreamPlan& plan, const CUtensorMap& map, const StreamParams& prm,
                    int64_t b, cudaStream_t stream) {
-  auto kern = gemv_stream_kernel<M_T>;
+  auto kern = gemv_stream_kernel<M_T, kClusterK>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [&] {
@@ -386,11 +428,19 @@ cudaError_t launch(const StreamPlan& plan, const CUtensorMap& map, const StreamP
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = plan.smem_bytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  int num_attrs = 1;
+  if (plan.cluster_k) {
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)plan.split_k;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    num_attrs = 2;
+  }
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = num_attrs;
   return cudaLaunchKernelEx(&cfg, kern, map, prm);
 }
 
@@ -403,27 +453,40 @@ bool stream_shape_supported(int64_t b, int m, int64_t k, int64_t n, const void* 
   return true;
 }
 
-StreamPlan stream_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int split_k) {
+// `split_k` 0: by shape.  `scratch_reduce`: keep the slices' sums in scratch and add them with
+// the reduce kernel even where a cluster could (for tests and comparisons).
+StreamPlan stream_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int split_k, bool scratch_reduce) {
   StreamPlan pl{};
   pl.m_tile = m <= 1 ? 1 : m <= 2 ? 2 : 4;
   pl.strips = (int)((n + kStripCols - 1) / kStripCols);
   const int64_t blocks = b * pl.strips;
+  const int slice_cap = max_slice_k(pl.m_tile);
+  const int64_t max_s = (k + kBoxRows - 1) / kBoxRows;           // at least one box per slice
+  const int64_t min_s = (k + slice_cap - 1) / slice_cap;         // the staged part of A must fit
   int64_t s = split_k;
   if (s <= 0) {
-    // Two blocks per SM keep enough loads in flight; more slices only add reduce traffic.
+    // Two blocks per SM keep enough loads in flight; more slices only add reduce work.  The
+    // planner's own choice is a power of two up to 8, so that the slices of a strip form a
+    // cluster (the portable size limit) and pack the GPCs without leftovers.
     s = 1;
-    if (blocks * 10 < (int64_t)sms * 13) s = std::min<int64_t>((2 * sms + blocks - 1) / blocks, k / 512);
+    if (blocks * 10 < (int64_t)sms * 13) {
+      const int64_t want = std::min<int64_t>((2 * sms + blocks - 1) / blocks, k / 512);
+      while (s * 2 <= want && s * 2 <= kMaxClusterK) s *= 2;
+    }
+    while (s < min_s && s < kMaxClusterK) s *= 2;
   }
-  const int slice_cap = max_slice_k(pl.m_tile);
-  s = std::max<int64_t>(s, (k + slice_cap - 1) / slice_cap);
-  s = std::max<int64_t>(1, std::min<int64_t>(s, (k + kBoxRows - 1) / kBoxRows));
+  s = std::max<int64_t>(s, min_s);
+  s = std::max<int64_t>(1, std::min<int64_t>(s, max_s));
   int64_t kps = (k + s - 1) / s;
   kps = (kps + kBoxRows - 1) / kBoxRows * kBoxRows;
   pl.k_per_split = (int)kps;
   pl.split_k = (int)((k + kps - 1) / kps);
   pl.supported = kps <= slice_cap;
+  // Up to 8 slices are added inside a cluster; more (a forced split, or a k too long for 8
+  // slices) go through scratch and the reduce kernel.
+  pl.cluster_k = !scratch_reduce && pl.split_k > 1 && pl.split_k <= kMaxClusterK;
   pl.smem_bytes = smem_for(pl.m_tile, pl.k_per_split);
-  pl.workspace_bytes = pl.split_k > 1 ? (size_t)pl.split_k * b * m * n * 4 : 0;
+  pl.workspace_bytes = (pl.split_k > 1 && !pl.cluster_k) ? (size_t)pl.split_k * b * m * n * 4 : 0;
   return pl;
 }
 
@@ -439,6 +502,7 @@ cudaError_t stream_launch(const DeviceInfo& dev, const StreamPlan& plan, int64_t
   prm.m = m;
   prm.strips = plan.strips;
   prm.split_k = plan.split_k;
+  prm.cluster_k = plan.cluster_k ? 1 : 0;
   prm.k_per_split = plan.k_per_split;
   prm.a_bulk = (k % 8 == 0 && reinterpret_cast<uintptr_t>(A) % 16 == 0 && a_batch % 8 == 0) ? 1 : 0;
   prm.status = dev.status;
@@ -451,15 +515,18 @@ cudaError_t stream_launch(const DeviceInfo& dev, const StreamPlan& plan, int64_t
     prm.A = A + b0 * a_batch;
     prm.C = C + b0 * c_batch;
     prm.partial = workspace ? workspace + b0 * m * n : nullptr;
-    switch (plan.m_tile) {
-      case 1: e = launch<1>(plan, map, prm, bn, stream); break;
-      case 2: e = launch<2>(plan, map, prm, bn, stream); break;
-      default: e = launch<4>(plan, map, prm, bn, stream); break;
+    switch (plan.m_tile * 2 + (plan.cluster_k ? 1 : 0)) {
+      case 2: e = launch<1, false>(plan, map, prm, bn, stream); break;
+      case 3: e = launch<1, true>(plan, map, prm, bn, stream); break;
+      case 4: e = launch<2, false>(plan, map, prm, bn, stream); break;
+      case 5: e = launch<2, true>(plan, map, prm, bn, stream); break;
+      case 8: e = launch<4, false>(plan, map, prm, bn, stream); break;
+      default: e = launch<4, true>(plan, map, prm, bn, stream); break;
     }
     if (e != cudaSuccess) return e;
     ++*launches;
   }
-  if (plan.split_k > 1) {
+  if (plan.split_k > 1 && !plan.cluster_k) {
     cudaError_t e = skinny_reduce_launch(workspace, C, b, m, n, c_batch, plan.split_k, stream, overwrite);
     if (e != cudaSuccess) return e;
     ++*launches;

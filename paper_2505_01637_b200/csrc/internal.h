@@ -58,13 +58,16 @@ struct StreamPlan {
   int m_tile;        // 1, 2 or 4
   int strips;        // thread blocks along n (64 columns each)
   int split_k;       // thread blocks along k
-  int k_per_split;   // multiple of 64
+  int k_per_split;   // multiple of the box height
+  bool cluster_k;    // the slices of a strip are one cluster and add up through distributed
+                     // shared memory: one launch, no scratch (2 <= split_k <= 8)
   size_t smem_bytes;
-  size_t workspace_bytes;  // partial sums [split_k][b][m][n] f32 when split_k > 1
+  size_t workspace_bytes;  // partial sums [split_k][b][m][n] f32 when the reduce kernel adds them
 };
 // Needs n % 8 == 0 and a 16-byte-aligned B (the TMA engine addresses B through a tensor map).
 bool stream_shape_supported(int64_t b, int m, int64_t k, int64_t n, const void* B);
-StreamPlan stream_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int split_k);
+StreamPlan stream_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int split_k,
+                       bool scratch_reduce = false);
 cudaError_t stream_launch(const DeviceInfo& dev, const StreamPlan& plan, int64_t b, int m, int64_t k,
                           int64_t n, const uint16_t* A, int64_t a_batch, const uint16_t* B, float* C,
                           int64_t c_batch, float* workspace, cudaStream_t stream,

@@ -134,12 +134,27 @@ def test_stream_kernel_matches_oracle(shape):
     check_full(A, B, C, integer=False, path=mb.MORELLO_PATH_SKINNY, split_k=STREAM, what="stream %s" % (shape,))
 
 
-@pytest.mark.parametrize("split_k", [1, 2, 3, 7, 32])
-def test_stream_kernel_forced_splits(split_k):
+@pytest.mark.parametrize("split_k", [1, 2, 3, 7, 8, 32])
+@pytest.mark.parametrize("kernel", [STREAM, STREAM + 1024])     # slices added in a cluster / from scratch
+def test_stream_kernel_forced_splits(split_k, kernel):
     for (b, m, k, n) in [(1, 1, 2048, 256), (2, 3, 1000, 72), (1, 4, 4096, 64)]:
         A, B, C = w.make(b, m, k, n, seed=split_k, ab="int4", c="normal")
-        check_full(A, B, C, integer=True, path=mb.MORELLO_PATH_SKINNY, split_k=STREAM + split_k,
-                   what="stream split %d %s" % (split_k, (b, m, k, n)))
+        got = check_full(A, B, C, integer=True, path=mb.MORELLO_PATH_SKINNY, split_k=kernel + split_k,
+                         what="stream split %d %s" % (split_k, (b, m, k, n)))
+        A, B, C = w.make(b, m, k, n, seed=split_k + 1, ab="uniform", c="normal")
+        check_full(A, B, C, integer=False, path=mb.MORELLO_PATH_SKINNY, split_k=kernel + split_k)
+
+
+def test_stream_kernel_cluster_reduce_needs_no_scratch_and_repeats():
+    b, m, k, n = 1, 1, 16384, 2048          # few strips, long k: eight slices per strip, one cluster each
+    assert mb.morello_workspace_bytes_forced(mb.MORELLO_PATH_SKINNY, STREAM, b, m, k, n) == 0
+    assert mb.morello_workspace_bytes_forced(mb.MORELLO_PATH_SKINNY, STREAM + 1024, b, m, k, n) > 0
+    A, B, C = w.make(b, m, k, n, seed=77, ab="int4", c="normal")
+    check_full(A, B, C, integer=True, path=mb.MORELLO_PATH_SKINNY, split_k=STREAM, what="cluster reduce")
+    A, B, C = w.make(b, m, k, n, seed=78, ab="uniform", c="normal")
+    first = gpu_run(A, B, C, path=mb.MORELLO_PATH_SKINNY, split_k=STREAM, calls=3)
+    again = gpu_run(A, B, C, path=mb.MORELLO_PATH_SKINNY, split_k=STREAM, calls=3)
+    assert np.array_equal(bits(first), bits(again))
 
 
 def test_stream_kernel_one_hot_and_repeatability():
