@@ -189,9 +189,8 @@ size_t morello_noalloc_scratch_limit(void);
 /* The path the selector picks for this shape with 16-byte-aligned operands:
  * MORELLO_PATH_SKINNY or MORELLO_PATH_TCGEN05 (-1 for an invalid shape).  A single row
  * (the GEMV) goes to the FP32-FMA kernels; from 2 rows on the tcgen05 kernels run whenever they can
- * address the shape (k % 8 == 0, n % 8 == 0) and, up to 16 rows, B has enough columns
- * to give half the SMs a tile (the choice uses the current device's SM count, 148 when
- * no device is usable). */
+ * address the shape (k % 8 == 0, n % 8 == 0).  (Nothing in the choice depends on the device;
+ * 148 SMs are assumed when no device is usable). */
 int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n);
 
 /*
@@ -205,8 +204,8 @@ int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n);
  * with the slices always added by the reduce kernel from scratch.  On the tcgen05 path, which never
  * splits k, the argument instead selects the tile: (value % 16) is the form -- 0 = by
  * shape, 1 = one CTA per 128-row tile, 2 = a pair of CTAs per 256-row tile
- * (cta_group::2), 3 = the operand-swapped kernel for at most 64 rows (no column count
- * with it) -- ((value / 16) % 16) is the tile's column count / 64 -- 0 = by
+ * (cta_group::2), 3 = the operand-swapped kernel for at most 64 rows (with it the next
+ * field is the number of k slices added inside a cluster instead: 0 = by shape, 1, 2, 4, 8) -- ((value / 16) % 16) is the tile's column count / 64 -- 0 = by
  * shape, 1, 2 or 4 (64 columns only with form 1) -- and adding 256 keeps the tiles of a
  * sparse last wave whole instead of cutting them into column halves.  Returns MORELLO_ERR_UNSUPPORTED_PATH, and
  * enqueues nothing, when the path cannot run the shape (the tcgen05 path needs

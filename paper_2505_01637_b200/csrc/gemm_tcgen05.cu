@@ -415,6 +415,8 @@ struct SwapParams {
   int64_t m, n;
   int64_t c_batch;  // m * n
   int k_blocks;
+  int split_k;      // k slices per strip (cluster form: the slices of a strip are one cluster)
+  int kb_per_slice; // k blocks per slice
   uint32_t* status;
 };
 
@@ -426,7 +428,12 @@ struct SwapBarriers {
   int abort_flag;
 };
 
-template <int kRowsA>
+// kClusterK: few strips and a long k -- the k range is cut into 2, 4 or 8 slices, the blocks
+// of a strip form a thread-block cluster, each parks its accumulator in its own shared memory
+// (the stage ring is free by then) and the blocks share the rows out among themselves: each adds
+// its rows' slices through distributed shared memory in slice order, then C: one launch, no
+// scratch, a fixed order.
+template <int kRowsA, bool kClusterK>
 __global__ void __launch_bounds__(kThreads)
 swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const SwapParams p) {
@@ -439,8 +446,12 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int col0 = blockIdx.x * kSwapStripCols;
+  const int strip = kClusterK ? blockIdx.x / p.split_k : blockIdx.x;
+  const int slice = kClusterK ? blockIdx.x % p.split_k : 0;     // = rank in the cluster
+  const int col0 = strip * kSwapStripCols;
   const int bb = blockIdx.y;
+  const int kb_begin = kClusterK ? slice * p.kb_per_slice : 0;
+  const int kb_end = kClusterK ? min(p.k_blocks, kb_begin + p.kb_per_slice) : p.k_blocks;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S::kStages; ++s) {
@@ -452,8 +463,8 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     mbar_fence_init();
     tma_prefetch_descriptor(&map_a);
     tma_prefetch_descriptor(&map_b);
-    const int ahead = min(p.k_blocks, kSwapPrefetchBlocks);
-    for (int kb = 0; kb < ahead; ++kb) {
+    const int ahead = min(kb_end, kb_begin + kSwapPrefetchBlocks);
+    for (int kb = kb_begin; kb < ahead; ++kb) {
       if (p.bt) {
         tma_prefetch_l2_3d(&map_b, kb * kTileK, col0, bb);
         tma_prefetch_l2_3d(&map_b, kb * kTileK, col0 + 64, bb);
@@ -481,7 +492,7 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     if (elect_one()) {
       int stage = 0;
       uint32_t phase = 0;
-      for (int kb = 0; kb < p.k_blocks; ++kb) {
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
         if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag, p.status, 8)) break;
         uint8_t* sb = stages + (size_t)stage * S::kStageBytes;
         uint8_t* sa = sb + S::kBytesStrip;
@@ -509,7 +520,7 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int kb = 0; kb < p.k_blocks; ++kb) {
+      for (int kb = kb_begin; kb < kb_end; ++kb) {
         if (!(ok = mbar_wait(&bars->full[stage], phase, abort_flag, p.status, 9))) break;
         tc_fence_after_sync();
         const uint32_t sb = smem_u32(stages + (size_t)stage * S::kStageBytes);
@@ -522,7 +533,7 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           const uint64_t d_strip = p.bt ? smem_desc_sw128(sb + j * 32, 16, 1024)
                                         : smem_desc_sw128(sb + j * 2048, kBoxBytesB, 1024);
           const uint64_t d_rows = smem_desc_sw128(sa + j * 32, 16, 1024);
-          mma_bf16_ss(tmem_base, d_strip, d_rows, idesc, (kb | j) != 0 ? 1u : 0u);
+          mma_bf16_ss(tmem_base, d_strip, d_rows, idesc, ((kb - kb_begin) | j) != 0 ? 1u : 0u);
         }
         mma_commit(&bars->empty[stage]);
         if (++stage == S::kStages) { stage = 0; phase ^= 1; }
@@ -535,25 +546,63 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const int64_t col = (int64_t)col0 + quarter * 32 + lane;   // this thread's column of C
     const bool col_live = col < p.n;
     float* c_col = p.C + (int64_t)bb * p.c_batch + col;
+    // Cluster form: block r of the cluster finishes the rows i with i % split_k == r.
     float c_in[kRowsA];
 #pragma unroll
-    for (int i = 0; i < kRowsA; ++i)
-      c_in[i] = (col_live && i < p.m && !p.overwrite) ? c_col[(int64_t)i * p.n] : 0.f;
+    for (int i = 0; i < kRowsA; ++i) {
+      const bool mine = !kClusterK || (i % p.split_k) == slice;
+      c_in[i] = (mine && col_live && i < p.m && !p.overwrite) ? c_col[(int64_t)i * p.n] : 0.f;
+    }
     bool ok = mbar_wait(&bars->acc_full, 0, abort_flag, p.status, 10);
     ok = __all_sync(0xffffffffu, ok);  // also reconverges the warp for the aligned TMEM loads
     if (ok) {
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+      // Cluster form: every MMA has completed, so the stage ring is free; the accumulator is
+      // parked there as part[row][128 columns of the strip].
+      float* part = reinterpret_cast<float*>(stages);
 #pragma unroll
       for (int g = 0; g < kRowsA / 16; ++g) {
         uint32_t r[16];
         tmem_ld_32x16(taddr + g * 16, r);
         tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 16; ++i)
-          if (col_live && g * 16 + i < p.m)
-            c_col[(int64_t)(g * 16 + i) * p.n] = c_in[g * 16 + i] + __uint_as_float(r[i]);
+        for (int i = 0; i < 16; ++i) {
+          if constexpr (kClusterK) {
+            part[(g * 16 + i) * kSwapStripCols + quarter * 32 + lane] = __uint_as_float(r[i]);
+          } else {
+            if (col_live && g * 16 + i < p.m)
+              c_col[(int64_t)(g * 16 + i) * p.n] = c_in[g * 16 + i] + __uint_as_float(r[i]);
+          }
+        }
       }
+    }
+    if constexpr (kClusterK) {
+      // Both cluster barriers are executed by every thread of every block (see below); between
+      // them every block finishes its share of the rows: the slices' sums in slice order (read
+      // through distributed shared memory), then C, then the store.
+      __syncwarp();
+      cluster_sync();
+      if (!*abort_flag) {
+        const float* part = reinterpret_cast<const float*>(stages);
+#pragma unroll
+        for (int i = 0; i < kRowsA; ++i) {
+          if (!col_live || i >= p.m || (i % p.split_k) != slice) continue;
+          const float* mine = part + i * kSwapStripCols + quarter * 32 + lane;
+          float sum = *peer_shared(mine, 0u);
+          for (int s2 = 1; s2 < p.split_k; ++s2) sum += *peer_shared(mine, (uint32_t)s2);
+          c_col[(int64_t)i * p.n] = c_in[i] + sum;
+        }
+      }
+      __syncwarp();
+      cluster_sync();
+    }
+  }
+  if constexpr (kClusterK) {
+    if (warp < 2) {        // producer and MMA warps take part in the two cluster barriers too
+      __syncwarp();
+      cluster_sync();
+      cluster_sync();
     }
   }
 
@@ -711,24 +760,43 @@ int gemm_pair_units(int sms) { return pair_units(sms); }
 // pair), weighted by what the narrower and the one-CTA tiles were measured to cost per
 // column (they re-read A more often, and a lone CTA reads the whole B tile from its own
 // shared memory).
-GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t, int64_t n, int knob) {
+GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob) {
   const bool halves = (knob / 256) == 0;
   knob %= 256;
   int form = knob % 16, tile_n = (knob / 16) * 64;
-  // Form 3: the operand-swapped kernel.  By shape it takes every call of at most 64 rows whose
-  // strips of 128 columns occupy at least half the SMs (measured on 2048 x 16384, us per call,
-  // swapped / 128-row tiles: m = 16: 11.7 / 14.2, 32: 12.6 / 14.4, 48: 13.1 / 14.6, 64: 13.8 / 14.9).
-  // Beyond 64 rows the 128-row tiles win: an accumulator of more than 64 columns per thread
-  // cannot be paired with an early read of C in registers, and sending the sums out as L2
-  // reductions instead cost more than it saved (96 rows: 16.7 against 15.4 us).
-  if (form == 3 || (form == 0 && tile_n == 0 && m <= kSwapMaxRows && b <= 65535 &&
-                    b * ((n + kSwapStripCols - 1) / kSwapStripCols) * 2 >= sms)) {
-    if (m > kSwapMaxRows || tile_n != 0 || b > 65535) return GemmPlan{false, 0, 0, 0, false};
-    return GemmPlan{true, 3, a_box_rows(m), 0, false};
+  // Form 3: the operand-swapped kernel.  By shape it takes every call of at most 64 rows
+  // (measured on 2048 x 16384, us per call, swapped / 128-row tiles: m = 16: 11.7 / 14.2, 32:
+  // 12.6 / 14.4, 48: 13.1 / 14.6, 64: 13.8 / 14.9; with few columns it wins as well: 16 x 4096 x
+  // 4096: 14.4 / 16.0).  Beyond 64 rows the 128-row tiles win: an accumulator of more than 64
+  // columns per thread cannot be paired with an early read of C in registers, and sending the
+  // sums out as L2 reductions instead cost more than it saved (96 rows: 16.7 against 15.4 us).
+  if (form == 3 || (form == 0 && tile_n == 0 && m <= kSwapMaxRows && b <= 65535)) {
+    // With form 3 the knob's column field is the number of k slices instead (0 = by shape).
+    const int forced_split = tile_n / 64;
+    if (m > kSwapMaxRows || b > 65535 ||
+        (forced_split != 0 && forced_split != 1 && forced_split != 2 && forced_split != 4 && forced_split != 8))
+      return GemmPlan{false, 0, 0, 0, false, 1};
+    const int64_t strips = b * ((n + kSwapStripCols - 1) / kSwapStripCols);
+    const int64_t k_blocks = (k + kTileK - 1) / kTileK;
+    int split = forced_split;
+    if (split == 0) {
+      // Few strips and a long k: cut k.  Measured (us per call, 1 / 2 / 4 / 8 slices): 16 rows,
+      // 16 strips (16384 x 2048): 48 / 31 / 19 / 15; 32 strips (4096 x 4096): 14.4 / 13.4 / 11.1 /
+      // 10.3; 64 strips (4096 x 8192): 15.6 / 16.5; 128 strips (2048 x 16384): 11.8 / 15.9.  With
+      // more than 16 rows a block fills an SM and clusters of them pack badly (48 rows, 16
+      // strips: 14.2 / 24.1 / 19.3).  So: up to 16 rows and up to 32 strips, as many slices as
+      // leave four k blocks each.
+      split = 1;
+      (void)sms;
+      if (a_box_rows(m) == 16 && strips <= 32)
+        while (split < 8 && k_blocks >= 8 * split) split *= 2;
+    }
+    while (split > 1 && (k_blocks + split - 1) / split * (split - 1) >= k_blocks) split /= 2;   // no empty slice
+    return GemmPlan{true, 3, a_box_rows(m), 0, false, split};
   }
   if (form < 0 || form > 2 || (tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) ||
       (form == 2 && tile_n == 64))
-    return GemmPlan{false, 0, 0, 0, false};
+    return GemmPlan{false, 0, 0, 0, false, 1};
   double best = 0;
   int best_form = 0, best_n = 0;
   if (form != 2 && tile_n == 0 && m <= kRowsPerCta) {
@@ -736,7 +804,7 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t, int64_t n, int knob) 
     best_n = 64;
     for (int tn = 256; tn >= 64; tn >>= 1)
       if (b * ((n + tn - 1) / tn) * 5 >= (int64_t)sms * 4) { best_n = tn; break; }
-    return GemmPlan{true, best_form, best_n, 0, halves};
+    return GemmPlan{true, best_form, best_n, 0, halves, 1};
   }
   for (int f = 1; f <= 2; ++f) {
     if (form != 0 && f != form) continue;
@@ -756,8 +824,8 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t, int64_t n, int knob) 
       if (best_n == 0 || cost < best) { best = cost; best_form = f; best_n = tn; }
     }
   }
-  if (best_n == 0) return GemmPlan{false, 0, 0, 0, false};
-  return GemmPlan{true, best_form, best_n, 0, halves};
+  if (best_n == 0) return GemmPlan{false, 0, 0, 0, false, 1};
+  return GemmPlan{true, best_form, best_n, 0, halves, 1};
 }
 
 namespace {
@@ -821,16 +889,16 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
 
 namespace {
 
-template <int kRowsA>
-cudaError_t launch_swap(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, int64_t n,
-                        const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
-                        bool overwrite, bool bt, cudaStream_t stream, uint64_t* launches) {
+template <int kRowsA, bool kClusterK>
+cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_t m, int64_t k, int64_t n,
+                             const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
+                             bool overwrite, bool bt, cudaStream_t stream, uint64_t* launches) {
   using S = SwapShape<kRowsA>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(swap_kernel<kRowsA>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)S::kSmemBytes);
+    attr_err = cudaFuncSetAttribute(swap_kernel<kRowsA, kClusterK>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::kSmemBytes);
   });
   if (attr_err != cudaSuccess) return attr_err;
   SwapParams p{};
@@ -839,6 +907,8 @@ cudaError_t launch_swap(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   p.m = m; p.n = n;
   p.c_batch = m * n;
   p.k_blocks = (int)((k + kTileK - 1) / kTileK);
+  p.split_k = kClusterK ? split : 1;
+  p.kb_per_slice = (p.k_blocks + p.split_k - 1) / p.split_k;
   p.status = dev.status;
   const int64_t strips = (n + kSwapStripCols - 1) / kSwapStripCols;
   // grid.y carries the batch index (the planner keeps batches beyond a grid dimension off
@@ -846,19 +916,37 @@ cudaError_t launch_swap(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   if (b > 65535) return cudaErrorInvalidValue;
   p.C = C;
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3((unsigned)strips, (unsigned)b, 1);
+  cfg.gridDim = dim3((unsigned)(strips * p.split_k), (unsigned)b, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = S::kSmemBytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  int num_attrs = 1;
+  if (kClusterK) {
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)p.split_k;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    num_attrs = 2;
+  }
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, swap_kernel<kRowsA>, map_a, map_b, p);
+  cfg.numAttrs = num_attrs;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, swap_kernel<kRowsA, kClusterK>, map_a, map_b, p);
   if (e != cudaSuccess) return e;
   ++*launches;
   return cudaSuccess;
+}
+
+template <int kRowsA>
+cudaError_t launch_swap(const DeviceInfo& dev, int split, int64_t b, int64_t m, int64_t k, int64_t n,
+                        const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
+                        bool overwrite, bool bt, cudaStream_t stream, uint64_t* launches) {
+  return split > 1 ? launch_swap_form<kRowsA, true>(dev, split, b, m, k, n, map_a, map_b, C, overwrite,
+                                                    bt, stream, launches)
+                   : launch_swap_form<kRowsA, false>(dev, 1, b, m, k, n, map_a, map_b, C, overwrite, bt,
+                                                     stream, launches);
 }
 
 }  // namespace
@@ -871,10 +959,10 @@ cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, 
   if (e != cudaSuccess) return e;
   const int code = plan.form * 1000 + plan.tile_n;
   switch (code) {
-    case 3016: return launch_swap<16>(dev, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
-    case 3032: return launch_swap<32>(dev, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
-    case 3048: return launch_swap<48>(dev, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
-    case 3064: return launch_swap<64>(dev, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
+    case 3016: return launch_swap<16>(dev, plan.split_k, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
+    case 3032: return launch_swap<32>(dev, plan.split_k, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
+    case 3048: return launch_swap<48>(dev, plan.split_k, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
+    case 3064: return launch_swap<64>(dev, plan.split_k, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
     case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, bt, stream); break;
     case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, bt, stream); break;
     case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, bt, stream); break;

@@ -340,7 +340,7 @@ gemv_stream_kernel(const __grid_constant__ CUtensorMap map_b, const StreamParams
         const int64_t col = col0 + (o % kStripCols);
         if (o >= M_T * kStripCols || i >= p.m || col >= p.n) continue;
         float sum = sums[r];
-        for (int s2 = 1; s2 < p.split_k; ++s2) sum += ld_shared_cluster_f32(map_to_cta(smem_u32(out_s + o), s2));
+        for (int s2 = 1; s2 < p.split_k; ++s2) sum += *peer_shared(out_s + o, (uint32_t)s2);
         p.C[(int64_t)bb * p.c_batch + (int64_t)i * p.n + col] = c_in[r] + sum;
       }
     }

@@ -88,12 +88,14 @@ struct GemmPlan {
   int tile_n;    // 64, 128 or 256 columns per tile
   size_t workspace_bytes;
   bool halves;   // tiles of a sparse last wave may be cut into column halves
+  int split_k;   // operand-swapped kernel only: k slices per strip, added inside a cluster (1, 2, 4, 8)
 };
 
 bool gemm_shape_supported(int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
                           const void* B, const void* C);
 // `knob`: 0 = by shape; otherwise form + 16 * (tile columns / 64) [+ 256 to keep the last wave's
-// tiles whole], the first two parts 0 = by shape.
+// tiles whole], the first two parts 0 = by shape; with form 3 the second part is the number of k
+// slices (0 = by shape, 1, 2, 4 or 8).
 GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob);
 // CTA pairs (cta_group::2) the current device can hold at once.
 int gemm_pair_units(int sms);

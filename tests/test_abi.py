@@ -67,8 +67,9 @@ def test_selector_is_shape_based(mb):
     assert mb.morello_select_path(1, 4, 4, 16) == mb.MORELLO_PATH_SKINNY
     assert mb.morello_select_path(1, 16, 2048, 16384) == mb.MORELLO_PATH_TCGEN05   # measured crossover: 2 rows
     assert mb.morello_select_path(1, 2, 2048, 16384) == mb.MORELLO_PATH_TCGEN05
-    assert mb.morello_select_path(1, 2, 2048, 1024) == mb.MORELLO_PATH_SKINNY      # too few column tiles
-    assert mb.morello_select_path(1, 16, 4096, 64) == mb.MORELLO_PATH_SKINNY        # too few column tiles
+    assert mb.morello_select_path(1, 2, 2048, 1024) == mb.MORELLO_PATH_TCGEN05     # few columns: k is cut instead
+    assert mb.morello_select_path(1, 16, 4096, 64) == mb.MORELLO_PATH_TCGEN05
+    assert mb.morello_select_path(1, 16, 4096, 60) == mb.MORELLO_PATH_SKINNY        # n % 8 != 0: TMA cannot address it
     assert mb.morello_select_path(1, 4096, 4096, 4095) == mb.MORELLO_PATH_SKINNY   # n % 8 != 0
     assert mb.morello_select_path(1, 4096, 4096, 4096) == mb.MORELLO_PATH_TCGEN05
     assert mb.morello_select_path(8, 2048, 2048, 16384) == mb.MORELLO_PATH_TCGEN05

@@ -32,6 +32,7 @@ CASES = [
     (0, (1, 16, 2048, 4096)),
     (3, (2, 5, 200, 264)),       # operand-swapped kernel, ragged
     (3, (1, 33, 72, 136)),
+    (3 + 16 * 8, (1, 16, 4096, 264)),   # ... eight k slices in a cluster
     (1, (1, 100, 72, 200)),      # one-CTA tiles, ragged
     (16 + 1, (1, 200, 136, 72)),
     (2, (2, 300, 520, 776)),     # CTA-pair tiles, ragged

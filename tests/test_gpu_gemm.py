@@ -175,6 +175,35 @@ def test_swap_form_one_hot_operands_and_repeatability():
     assert_bit_exact(gpu_run(A, B, C, path=TC, split_k=SWAP, calls=2), twice, "swap form, two accumulating calls")
 
 
+@pytest.mark.parametrize("slices", [2, 4, 8])
+@pytest.mark.parametrize("shape", [
+    (1, 16, 16384, 2048),   # the transposed weight shape: 16 strips, long k
+    (2, 3, 1000, 136),      # ragged k blocks, ragged strip, batches
+    (1, 64, 4096, 256),     # 64 rows: the accumulator parked in shared memory is 32 KiB
+    (1, 33, 520, 392),
+])
+def test_swap_form_with_k_slices_in_a_cluster(shape, slices):
+    b, m, k, n = shape
+    knob = SWAP + 16 * slices
+    A, B, C = w.make(b, m, k, n, seed=sum(shape) + slices, ab="int4", c="normal")
+    got = check_full(A, B, C, integer=True, path=TC, split_k=knob, what="swap, %d slices %s" % (slices, shape))
+    assert_bit_exact(gpu_run(A, B, C, path=TC, split_k=SWAP + 16), got, "slices vs one block per strip")
+    A, B, C = w.make(b, m, k, n, seed=sum(shape) + slices + 1, ab="uniform_rsqrtk", c="normal")
+    first = check_full(A, B, C, integer=False, path=TC, split_k=knob)
+    assert np.array_equal(bits(gpu_run(A, B, C, path=TC, split_k=knob)), bits(first))
+
+
+def test_swap_form_picks_slices_by_shape_and_refuses_odd_counts():
+    b, m, k, n = 1, 16, 8192, 1024          # 8 strips: the planner cuts k by itself
+    A, B, C = w.make(b, m, k, n, seed=3, ab="int4", c="int8")
+    check_full(A, B, C, integer=True, what="auto slices")
+    from gpu_util import to_dev
+    dA, dB, dC = to_dev(A, B, C)
+    with pytest.raises(mb.MorelloError) as e:
+        mb.morello_matmul_accum_forced(TC, SWAP + 16 * 3, b, m, k, n, dA, dB, dC)
+    assert e.value.status == mb.MORELLO_ERR_UNSUPPORTED_PATH
+
+
 def test_swap_form_refuses_more_than_64_rows():
     b, m, k, n = 1, 65, 64, 128
     A, B, C = w.make(b, m, k, n, seed=1)

@@ -22,6 +22,7 @@ CASES = [
     (SK, 2048 + 3, (2, 2, 1000, 264)),     # ... with k slices
     (TC, 3, (2, 16, 200, 264)),            # operand-swapped kernel
     (TC, 3, (1, 50, 136, 264)),            # ... the 200 KiB ring
+    (TC, 3 + 16 * 4, (1, 16, 2048, 264)),  # ... four k slices in a cluster
     (TC, 1, (1, 100, 72, 200)),            # one-CTA tiles, ragged
     (TC, 2, (2, 300, 520, 776)),           # CTA-pair tiles, ragged
     (TC, 64 + 2, (2, 1100, 72, 4504)),     # last wave cut into halves

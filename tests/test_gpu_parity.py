@@ -95,21 +95,27 @@ def test_forced_split_k_matches_oracle(split_k):
 
 
 def test_caller_workspace_and_its_size_check():
-    b, m, k, n = 1, 4, 8192, 64          # few columns, long k: the planner splits k
+    b, m, k, n = 1, 4, 8192, 64          # few columns, long k: the register-streaming kernel splits k
+    REG = 1024                           # that kernel, split by shape
     A, B, C = w.make(b, m, k, n, seed=5, ab="int4", c="normal")
-    need = mb.morello_workspace_bytes(b, m, k, n)
-    assert need > 0
+    need = mb.morello_workspace_bytes_forced(mb.MORELLO_PATH_SKINNY, REG, b, m, k, n)
+    assert need > 0 and mb.morello_workspace_bytes(b, m, k, n) >= need
     dA, dB, dC = to_dev(A, B, C)
     ws = torch.full((need // 4 + 64,), float("nan"), device="cuda")   # poisoned scratch
-    mb.morello_matmul_accum_ws(b, m, k, n, dA, dB, dC, ws, need)
-    assert_bit_exact(dC.cpu().numpy(), oracle.matmul_accum(b, m, k, n, A, B, C), "ws variant")
+    mb.morello_matmul_accum_forced(mb.MORELLO_PATH_SKINNY, REG, b, m, k, n, dA, dB, dC, ws, need)
+    assert_bit_exact(dC.cpu().numpy(), oracle.matmul_accum(b, m, k, n, A, B, C), "caller's scratch")
     assert torch.isnan(ws[need // 4:]).all()                          # nothing past the stated size
     before = dC.clone()
     with pytest.raises(mb.MorelloError) as e:
-        mb.morello_matmul_accum_ws(b, m, k, n, dA, dB, dC, ws, need - 4)
+        mb.morello_matmul_accum_forced(mb.MORELLO_PATH_SKINNY, REG, b, m, k, n, dA, dB, dC, ws, need - 4)
     assert e.value.status == mb.MORELLO_ERR_WORKSPACE
     torch.cuda.synchronize()
     assert torch.equal(before, dC)
+    # the selector's own choice for this shape needs no scratch at all; the _ws call takes any
+    dC2 = torch.from_numpy(C.copy()).cuda()
+    mb.morello_matmul_accum_ws(b, m, k, n, dA, dB, dC2, ws, need)
+    torch.cuda.synchronize()
+    assert_bit_exact(dC2.cpu().numpy(), oracle.matmul_accum(b, m, k, n, A, B, C), "ws variant")
 
 
 # ------------------------------------- T3b: the TMA-ring GEMV kernel, forced (knob 2048 + split)
