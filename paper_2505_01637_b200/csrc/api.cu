@@ -177,29 +177,16 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     return MORELLO_OK;
   }
 
+  bool bt_fallback = false;
   if (b_col_major) {
     // B as [b][n][k]: the tensor-core kernels when the TMA engine can address the operands,
     // else the one-warp-per-column kernel.  The FMA streaming kernels read B by rows only.
     if (path == MORELLO_PATH_SKINNY) return MORELLO_ERR_UNSUPPORTED_PATH;
     const bool tc = gemm_shape_supported(b, m, k, n, A, B, C);
     if (path == MORELLO_PATH_TCGEN05 && !tc) return MORELLO_ERR_UNSUPPORTED_PATH;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    uint64_t launches = 0;
-    cudaError_t e;
-    if (tc) {
-      const GemmPlan plan = gemm_plan(st->info.sms, b, m, k, n, split_k);
-      if (!plan.supported) return MORELLO_ERR_UNSUPPORTED_PATH;
-      e = gemm_launch(st->info, plan, b, m, k, n, static_cast<const uint16_t*>(A),
-                      static_cast<const uint16_t*>(B), C, nullptr, s, &launches, overwrite, true);
-    } else {
-      e = colmajor_fallback_launch(b, m, k, n, static_cast<const uint16_t*>(A),
-                                   static_cast<const uint16_t*>(B), C, overwrite, s, &launches);
-    }
-    g_launches.fetch_add(launches, std::memory_order_relaxed);
-    if (e != cudaSuccess) return cuda_fail(e);
-    return MORELLO_OK;
-  }
-  if (path == MORELLO_PATH_AUTO) {
+    path = MORELLO_PATH_TCGEN05;
+    bt_fallback = !tc;
+  } else if (path == MORELLO_PATH_AUTO) {
     path = select_path(st->info.sms, b, m, k, n, A, B, C);
   } else if (path == MORELLO_PATH_TCGEN05) {
     if (!gemm_shape_supported(b, m, k, n, A, B, C)) return MORELLO_ERR_UNSUPPORTED_PATH;
@@ -214,7 +201,7 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     which = skinny_kernel_for(split_k, b, m, k, n, B);
     if (which < 0) return MORELLO_ERR_UNSUPPORTED_PATH;
   }
-  const size_t need = workspace_for(sms, path, split_k, b, m, k, n, B);
+  const size_t need = bt_fallback ? 0 : workspace_for(sms, path, split_k, b, m, k, n, B);
   float* ws = static_cast<float*>(workspace);
   if (need > 0) {
     if (own_scratch) {
@@ -242,11 +229,14 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   uint64_t launches = 0;
   cudaError_t e = cudaSuccess;
-  if (path == MORELLO_PATH_TCGEN05) {
+  if (bt_fallback) {
+    e = colmajor_fallback_launch(b, m, k, n, static_cast<const uint16_t*>(A),
+                                 static_cast<const uint16_t*>(B), C, overwrite, s, &launches);
+  } else if (path == MORELLO_PATH_TCGEN05) {
     const GemmPlan plan = gemm_plan(sms, b, m, k, n, split_k);
     if (!plan.supported) return MORELLO_ERR_UNSUPPORTED_PATH;
     e = gemm_launch(st->info, plan, b, m, k, n, static_cast<const uint16_t*>(A),
-                    static_cast<const uint16_t*>(B), C, ws, s, &launches, overwrite);
+                    static_cast<const uint16_t*>(B), C, ws, s, &launches, overwrite, b_col_major);
   } else if (which == SKINNY_STREAM) {
     const StreamPlan plan = stream_plan(sms, b, (int)m, k, n, split_k % kKnobSplitMod,
                                         knob_scratch_reduce(split_k));

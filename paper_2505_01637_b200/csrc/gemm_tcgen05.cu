@@ -79,6 +79,11 @@ struct GemmParams {
   int64_t whole;    // work items [0, whole) are whole tiles, in tile order;
   int64_t items;    // items [whole, items) are the column halves of tiles [whole, tiles)
   int k_blocks;
+  int ws_split;     // > 1: few tiles and a long k -- every tile's k range is cut into this many
+                    // slices, each an item of its own whose sums go (as a plain store) to
+                    // partial[slice][b][m][n]; the slice-ordered reduce kernel adds them and C
+  int kb_per_slice; // k blocks per slice
+  int64_t bsz;      // batches
   uint32_t* status;
   int overwrite;   // 1: C = product (TMA store) instead of C += product (TMA reduce-add)
   int bt;          // 1: B is stored column-major, [b][n][k]: the K-major operand (boxes of 64 k x 64 columns)
@@ -99,6 +104,8 @@ struct Item {
   int mt, nt, bb;
   int n_off;   // first column of the item inside its tile
   int cols;    // columns of the item: the tile's width or half of it
+  int kb0, kb1;  // k blocks [kb0, kb1) of the item
+  int out_b;   // batch coordinate of the item's output in the map the epilogue stores through
 };
 template <int kTileN>
 __device__ __forceinline__ Item decode_item(const GemmParams& p, int64_t t) {
@@ -106,7 +113,15 @@ __device__ __forceinline__ Item decode_item(const GemmParams& p, int64_t t) {
   int64_t tile = t;
   it.n_off = 0;
   it.cols = kTileN;
-  if (t >= p.whole) {
+  it.kb0 = 0;
+  it.kb1 = p.k_blocks;
+  int slice = 0;
+  if (p.ws_split > 1) {            // items are (tile, slice); no halves in this mode
+    tile = t / p.ws_split;
+    slice = (int)(t - tile * p.ws_split);
+    it.kb0 = slice * p.kb_per_slice;
+    it.kb1 = min(p.k_blocks, it.kb0 + p.kb_per_slice);
+  } else if (t >= p.whole) {
     const int64_t h = t - p.whole;
     tile = p.whole + (h >> 1);
     it.cols = kTileN / 2;
@@ -115,6 +130,7 @@ __device__ __forceinline__ Item decode_item(const GemmParams& p, int64_t t) {
   it.mt = (int)(tile % p.m_tiles);
   it.nt = (int)((tile / p.m_tiles) % p.n_tiles);
   it.bb = (int)(tile / ((int64_t)p.m_tiles * p.n_tiles));
+  it.out_b = (int)(slice * p.bsz + it.bb);
   return it;
 }
 
@@ -199,7 +215,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int boxes_b = cols_b / 64;
         const int col0 = it.nt * kTileN + it.n_off + (int)rank * cols_b;
         const uint32_t stage_tx = (uint32_t)(boxes_b * kBoxBytesB + p.a_box_rows * (kTileK * 2));
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
+        for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!(ok = mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag, p.status, 1))) break;
           uint8_t* sa = stages + (size_t)stage * S::kStageBytes;
           uint8_t* sb = sa + kBytesA;
@@ -248,11 +264,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int64_t t = unit; t < p.items && ok; t += units) {
-        const uint32_t idesc = t < p.whole ? idesc_tile : idesc_half;
+        const Item it = decode_item<kTileN>(p, t);
+        const uint32_t idesc = it.cols == kTileN ? idesc_tile : idesc_half;
         if (!(ok = mbar_wait(&bars->acc_empty[buf], acc_phase ^ 1, abort_flag, p.status, 2))) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + (uint32_t)buf * kAccStride;
-        for (int kb = 0; kb < p.k_blocks; ++kb) {
+        for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!(ok = mbar_wait(&bars->full[stage], phase, abort_flag, p.status, 3))) break;
           tc_fence_after_sync();
           const uint32_t sa = smem_u32(stages + (size_t)stage * S::kStageBytes);
@@ -267,8 +284,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             // apart, 32 bytes per K step.)
             const uint64_t db = p.bt ? smem_desc_sw128(sb + j * 32, 16, 1024)
                                      : smem_desc_sw128(sb + j * 2048, kBoxBytesB, 1024);
-            if constexpr (kPair) mma_bf16_ss_pair(d_tmem, da, db, idesc, (kb | j) != 0 ? 1u : 0u);
-            else mma_bf16_ss(d_tmem, da, db, idesc, (kb | j) != 0 ? 1u : 0u);
+            const uint32_t accumulate = ((kb - it.kb0) | j) != 0 ? 1u : 0u;
+            if constexpr (kPair) mma_bf16_ss_pair(d_tmem, da, db, idesc, accumulate);
+            else mma_bf16_ss(d_tmem, da, db, idesc, accumulate);
           }
           // The stage is reusable (in both CTAs) once these MMAs have read it.
           if constexpr (kPair) mma_commit_pair(&bars->empty[stage], 3);
@@ -297,7 +315,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     for (int64_t t = unit; t < p.items && ok; t += units) {
       const Item it = decode_item<kTileN>(p, t);
       const int mt = it.mt;
-      const int bb = it.bb;
       ok = mbar_wait(&bars->acc_full[buf], acc_phase, abort_flag, p.status, 4);
       ok = __all_sync(0xffffffffu, ok);  // also reconverges the warp for the aligned TMEM loads
       if (!ok) break;
@@ -337,8 +354,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           if (lane == 0) {
             // C[bb, row0 : row0 + 32, col0 + c : col0 + c + 32] += block; rows and columns
             // past the edge of C are dropped by the TMA engine.
-            if (p.overwrite) tma_store_3d(&map_c, my_blocks + blk * kEpiBlockBytes, col0 + c, row0, bb);
-            else tma_reduce_add_3d(&map_c, my_blocks + blk * kEpiBlockBytes, col0 + c, row0, bb);
+            if (p.overwrite) tma_store_3d(&map_c, my_blocks + blk * kEpiBlockBytes, col0 + c, row0, it.out_b);
+            else tma_reduce_add_3d(&map_c, my_blocks + blk * kEpiBlockBytes, col0 + c, row0, it.out_b);
             bulk_commit_group();
           }
           blk ^= 1u;
@@ -415,7 +432,8 @@ struct SwapParams {
   int64_t m, n;
   int64_t c_batch;  // m * n
   int k_blocks;
-  int split_k;      // k slices per strip (cluster form: the slices of a strip are one cluster)
+  int split_k;      // k slices per strip (cluster form: the slices of a strip are one cluster;
+                    // otherwise every slice writes its own copy of the output, see the kernel)
   int kb_per_slice; // k blocks per slice
   uint32_t* status;
 };
@@ -446,12 +464,12 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int strip = kClusterK ? blockIdx.x / p.split_k : blockIdx.x;
-  const int slice = kClusterK ? blockIdx.x % p.split_k : 0;     // = rank in the cluster
+  const int strip = blockIdx.x / p.split_k;
+  const int slice = blockIdx.x % p.split_k;     // cluster form: = rank in the cluster
   const int col0 = strip * kSwapStripCols;
   const int bb = blockIdx.y;
-  const int kb_begin = kClusterK ? slice * p.kb_per_slice : 0;
-  const int kb_end = kClusterK ? min(p.k_blocks, kb_begin + p.kb_per_slice) : p.k_blocks;
+  const int kb_begin = slice * p.kb_per_slice;
+  const int kb_end = min(p.k_blocks, kb_begin + p.kb_per_slice);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S::kStages; ++s) {
@@ -545,7 +563,9 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const int quarter = warp & 3;  // TMEM lanes [32 * quarter, 32 * quarter + 32)
     const int64_t col = (int64_t)col0 + quarter * 32 + lane;   // this thread's column of C
     const bool col_live = col < p.n;
-    float* c_col = p.C + (int64_t)bb * p.c_batch + col;
+    // Without a cluster, slices > 1 means that C is partial[slice][b][m][n] in the workspace.
+    const int64_t out_b = kClusterK ? bb : (int64_t)slice * gridDim.y + bb;
+    float* c_col = p.C + out_b * p.c_batch + col;
     // Cluster form: block r of the cluster finishes the rows i with i % split_k == r.
     float c_in[kRowsA];
 #pragma unroll
@@ -623,9 +643,10 @@ struct MapKey {
   const void* c;
   int64_t bsz, m, k, n;
   bool bt;   // B column-major
+  int64_t c_bsz;   // batches of the output map: bsz, or slices x bsz when c is the workspace
   bool operator==(const MapKey& o) const {
     return a == o.a && b == o.b && c == o.c && bsz == o.bsz && m == o.m && k == o.k && n == o.n &&
-           bt == o.bt;
+           bt == o.bt && c_bsz == o.c_bsz;
   }
 };
 struct MapEntry {
@@ -672,7 +693,7 @@ cudaError_t get_maps(const MapKey& key, CUtensorMap* ma, CUtensorMap* mb, CUtens
                              CU_TENSOR_MAP_SWIZZLE_128B);
   if (err != cudaSuccess) return err;
   err = make_tensor_map_3d(&e.map_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, key.c, (uint64_t)key.n,
-                           (uint64_t)key.m, (uint64_t)key.bsz, kEpiCols, 32,
+                           (uint64_t)key.m, (uint64_t)key.c_bsz, kEpiCols, 32,
                            CU_TENSOR_MAP_SWIZZLE_128B);
   if (err != cudaSuccess) return err;
   e.stamp = ++g_stamp;
@@ -751,19 +772,63 @@ int pair_units(int sms) {
 
 int gemm_pair_units(int sms) { return pair_units(sms); }
 
-// The knob of the forced entry point (its split_k argument, which this path does not need:
-// k is never split) selects the tile: knob % 16 = form (0 by shape, 1 one CTA per tile,
-// 2 a CTA pair per tile), knob / 16 = tile columns / 64 (0 by shape; 1, 2 or 4).
+// The knob of the forced entry point (its split_k argument) selects the kernel and its tile:
+// knob % 16 = form (0 by shape, 1 one CTA per tile, 2 a CTA pair per tile, 3 operand-swapped),
+// (knob / 16) % 16 = tile columns / 64 (0 by shape; 1, 2 or 4; with form 3 the number of k slices
+// inside a cluster), + 256 keeps the last wave's tiles whole, (knob / 512) % 16 = k slices through
+// the workspace (0 by shape, 1 none, 2 .. 8).
+//
 // By shape: with a single row of tiles (m <= 128) the call streams B once and is bound by
 // memory, so the widest tile that still gives about one thread block per SM wins.  Otherwise
-// the candidate with the fewest "waves x columns" wins, a wave being one tile per SM (or per
-// pair), weighted by what the narrower and the one-CTA tiles were measured to cost per
-// column (they re-read A more often, and a lone CTA reads the whole B tile from its own
-// shared memory).
+// the candidate with the least "waves x k blocks x columns" wins, a wave being one tile per SM
+// (or per pair), weighted by what the narrower and the one-CTA tiles were measured to cost per
+// column (they re-read A more often, and a lone CTA reads the whole B tile from its own shared
+// memory).
+//
+// Few tiles and a long k: a call whose tiles fill less than half the device is cut along k as
+// well.  Each (tile, slice) item stores its sums to partial[slice][b][m][n] in the workspace
+// and one more launch adds the slices in slice order, then C -- the bits do not depend on which
+// block finished first.  (Measured, us per call before / after: 64 x 16384 x 2048: 46.5; 128 x
+// 16384 x 2048: 52.8; 512 x 16384 x 2048: 53.8.)
+namespace {
+
+constexpr int kWsMaxSplit = 8;
+constexpr int kWsMinBlocks = 16;                 // k blocks a slice keeps at least
+constexpr size_t kWsMaxBytes = size_t(64) << 20; // partial sums stay well inside L2
+
+// The largest number of k slices (<= want) whose partial sums fit the workspace cap and that
+// leaves no slice empty.
+int ws_fit(int want, int64_t k_blocks, int64_t b, int64_t m, int64_t n) {
+  int split = std::max(1, std::min(want, kWsMaxSplit));
+  while (split > 1 && (size_t)split * b * m * n * 4 > kWsMaxBytes) --split;
+  while (split > 1 && (k_blocks + split - 1) / split * (split - 1) >= k_blocks) --split;
+  return split;
+}
+
+}  // namespace
+
 GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob) {
-  const bool halves = (knob / 256) == 0;
+  if (knob < 0) return GemmPlan{false, 0, 0, 0, false, 1, 1};
+  const int forced_ws = (knob / 512) % 16;
+  const bool halves = ((knob / 256) % 2) == 0;
   knob %= 256;
   int form = knob % 16, tile_n = (knob / 16) * 64;
+  const int64_t k_blocks = (k + kTileK - 1) / kTileK;
+  if (forced_ws > kWsMaxSplit) return GemmPlan{false, 0, 0, 0, false, 1, 1};
+  auto finish = [&](GemmPlan plan) {
+    if (plan.ws_split > 1) {
+      plan.workspace_bytes = (size_t)plan.ws_split * b * m * n * 4;
+      plan.halves = false;
+    }
+    return plan;
+  };
+  // By shape, the k slices of `tiles` items on `units` units.
+  auto ws_by_shape = [&](int64_t tiles, int64_t units) {
+    if (forced_ws != 0) return ws_fit(forced_ws, k_blocks, b, m, n);
+    if (tiles * 2 > units || k_blocks < 2 * kWsMinBlocks) return 1;
+    const int64_t want = std::min<int64_t>(units / tiles, k_blocks / kWsMinBlocks);
+    return ws_fit((int)std::min<int64_t>(want, kWsMaxSplit), k_blocks, b, m, n);
+  };
   // Form 3: the operand-swapped kernel.  By shape it takes every call of at most 64 rows
   // (measured on 2048 x 16384, us per call, swapped / 128-row tiles: m = 16: 11.7 / 14.2, 32:
   // 12.6 / 14.4, 48: 13.1 / 14.6, 64: 13.8 / 14.9; with few columns it wins as well: 16 x 4096 x
@@ -775,9 +840,8 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob
     const int forced_split = tile_n / 64;
     if (m > kSwapMaxRows || b > 65535 ||
         (forced_split != 0 && forced_split != 1 && forced_split != 2 && forced_split != 4 && forced_split != 8))
-      return GemmPlan{false, 0, 0, 0, false, 1};
+      return GemmPlan{false, 0, 0, 0, false, 1, 1};
     const int64_t strips = b * ((n + kSwapStripCols - 1) / kSwapStripCols);
-    const int64_t k_blocks = (k + kTileK - 1) / kTileK;
     int split = forced_split;
     if (split == 0) {
       // Few strips and a long k: cut k.  Measured (us per call, 1 / 2 / 4 / 8 slices): 16 rows,
@@ -785,27 +849,30 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob
       // 10.3; 64 strips (4096 x 8192): 15.6 / 16.5; 128 strips (2048 x 16384): 11.8 / 15.9.  With
       // more than 16 rows a block fills an SM and clusters of them pack badly (48 rows, 16
       // strips: 14.2 / 24.1 / 19.3).  So: up to 16 rows and up to 32 strips, as many slices as
-      // leave four k blocks each.
+      // leave four k blocks each; the other shapes of few strips go through the workspace.
       split = 1;
-      (void)sms;
-      if (a_box_rows(m) == 16 && strips <= 32)
+      if (forced_ws <= 1 && a_box_rows(m) == 16 && strips <= 32)
         while (split < 8 && k_blocks >= 8 * split) split *= 2;
     }
     while (split > 1 && (k_blocks + split - 1) / split * (split - 1) >= k_blocks) split /= 2;   // no empty slice
-    return GemmPlan{true, 3, a_box_rows(m), 0, false, split};
+    int ws = 1;
+    if (split == 1) ws = ws_by_shape(strips, sms);
+    return finish(GemmPlan{true, 3, a_box_rows(m), 0, false, split, ws});
   }
   if (form < 0 || form > 2 || (tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) ||
       (form == 2 && tile_n == 64))
-    return GemmPlan{false, 0, 0, 0, false, 1};
-  double best = 0;
-  int best_form = 0, best_n = 0;
+    return GemmPlan{false, 0, 0, 0, false, 1, 1};
   if (form != 2 && tile_n == 0 && m <= kRowsPerCta) {
-    best_form = 1;
-    best_n = 64;
-    for (int tn = 256; tn >= 64; tn >>= 1)
-      if (b * ((n + tn - 1) / tn) * 5 >= (int64_t)sms * 4) { best_n = tn; break; }
-    return GemmPlan{true, best_form, best_n, 0, halves, 1};
+    int best_n = 64;
+    for (int tn = 256; tn >= 64; tn >>= 1) {
+      const int64_t tiles = b * ((n + tn - 1) / tn);
+      if (tiles * ws_by_shape(tiles, sms) * 5 >= (int64_t)sms * 4) { best_n = tn; break; }
+    }
+    const int64_t tiles = b * ((n + best_n - 1) / best_n);
+    return finish(GemmPlan{true, 1, best_n, 0, halves, 1, ws_by_shape(tiles, sms)});
   }
+  double best = 0;
+  int best_form = 0, best_n = 0, best_ws = 1;
   for (int f = 1; f <= 2; ++f) {
     if (form != 0 && f != form) continue;
     if (form == 0 && f == 2 && m <= kRowsPerCta) continue;   // a pair would idle its second CTA
@@ -814,18 +881,23 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob
       const int64_t tile_m = (int64_t)kRowsPerCta * f;
       const int64_t tiles = b * ((m + tile_m - 1) / tile_m) * ((n + tn - 1) / tn);
       const int64_t units = std::max(1, f == 2 ? pair_units(sms) : sms);
-      const int64_t tail = tiles % units;
-      const bool cut = halves && tiles > units && tail > 0 && 2 * tail <= units &&
+      const int ws = ws_by_shape(tiles, units);
+      const int64_t items = tiles * ws;
+      const int64_t tail = items % units;
+      const bool cut = ws == 1 && halves && tiles > units && tail > 0 && 2 * tail <= units &&
                        (tn / f / 2) % 64 == 0;
       // A last wave cut into halves costs about 0.6 of a whole one.
-      const double waves = (double)(tiles / units) + (tail == 0 ? 0.0 : cut ? 0.625 : 1.0);
-      const double cost = (double)waves * tn * (f == 1 ? 1.15 : 1.0) *
-                          (tn == 256 ? 1.0 : tn == 128 ? 1.25 : 1.6);
-      if (best_n == 0 || cost < best) { best = cost; best_form = f; best_n = tn; }
+      const double waves = (double)(items / units) + (tail == 0 ? 0.0 : cut ? 0.625 : 1.0);
+      // In units of one column of one k block on a pair's 256-column tile (about 1.5 ns).  The
+      // launch that adds the slices: about 3 us and its bytes at L2 speed.
+      double cost = waves * (double)((k_blocks + ws - 1) / ws) * tn * (f == 1 ? 1.15 : 1.0) *
+                    (tn == 256 ? 1.0 : tn == 128 ? 1.25 : 1.6);
+      if (ws > 1) cost += 2000.0 + (double)(ws + 2) * b * m * n * 4 / 4.5e3;
+      if (best_n == 0 || cost < best) { best = cost; best_form = f; best_n = tn; best_ws = ws; }
     }
   }
-  if (best_n == 0) return GemmPlan{false, 0, 0, 0, false, 1};
-  return GemmPlan{true, best_form, best_n, 0, halves, 1};
+  if (best_n == 0) return GemmPlan{false, 0, 0, 0, false, 1, 1};
+  return finish(GemmPlan{true, best_form, best_n, 0, halves, 1, best_ws});
 }
 
 namespace {
@@ -833,8 +905,8 @@ namespace {
 template <bool kPair, int kTileN>
 cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, int64_t n,
                         const CUtensorMap& map_a, const CUtensorMap& map_b,
-                        const CUtensorMap& map_c, float* C, bool halves, bool overwrite, bool bt,
-                        cudaStream_t stream) {
+                        const CUtensorMap& map_c, float* C, bool halves, int ws_split,
+                        bool overwrite, bool bt, cudaStream_t stream) {
   using S = Shape<kPair, kTileN>;
   const cudaError_t attr_err = set_smem_attribute<kPair, kTileN>();
   if (attr_err != cudaSuccess) return attr_err;
@@ -853,6 +925,15 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   p.a_box_rows = a_box_rows(m);
   p.overwrite = overwrite ? 1 : 0;
   p.bt = bt ? 1 : 0;
+  p.bsz = b;
+  p.ws_split = std::max(1, ws_split);
+  p.kb_per_slice = (p.k_blocks + p.ws_split - 1) / p.ws_split;
+  if (p.ws_split > 1) {      // map_c covers the partial sums; every item stores its own
+    p.items = p.tiles * p.ws_split;
+    p.whole = p.items;
+    p.overwrite = 1;
+    halves = false;
+  }
 
   const int64_t max_units = kPair ? pair_units(dev.sms) : dev.sms;
   // The last wave of a compute-bound problem: when its tiles would occupy at most half the
@@ -892,7 +973,7 @@ namespace {
 template <int kRowsA, bool kClusterK>
 cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_t m, int64_t k, int64_t n,
                              const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
-                             bool overwrite, bool bt, cudaStream_t stream, uint64_t* launches) {
+                             bool overwrite, bool bt, cudaStream_t stream) {
   using S = SwapShape<kRowsA>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
@@ -907,7 +988,7 @@ cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_
   p.m = m; p.n = n;
   p.c_batch = m * n;
   p.k_blocks = (int)((k + kTileK - 1) / kTileK);
-  p.split_k = kClusterK ? split : 1;
+  p.split_k = std::max(1, split);
   p.kb_per_slice = (p.k_blocks + p.split_k - 1) / p.split_k;
   p.status = dev.status;
   const int64_t strips = (n + kSwapStripCols - 1) / kSwapStripCols;
@@ -933,45 +1014,58 @@ cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_
   }
   cfg.attrs = attr;
   cfg.numAttrs = num_attrs;
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, swap_kernel<kRowsA, kClusterK>, map_a, map_b, p);
-  if (e != cudaSuccess) return e;
-  ++*launches;
-  return cudaSuccess;
+  return cudaLaunchKernelEx(&cfg, swap_kernel<kRowsA, kClusterK>, map_a, map_b, p);
 }
 
+// `split` > 1: the slices of a strip form a cluster and C is the output.  `ws_split` > 1: the
+// slices are independent blocks and C is the workspace, partial[slice][b][m][n].
 template <int kRowsA>
-cudaError_t launch_swap(const DeviceInfo& dev, int split, int64_t b, int64_t m, int64_t k, int64_t n,
-                        const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
-                        bool overwrite, bool bt, cudaStream_t stream, uint64_t* launches) {
+cudaError_t launch_swap(const DeviceInfo& dev, int split, int ws_split, int64_t b, int64_t m, int64_t k,
+                        int64_t n, const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
+                        bool overwrite, bool bt, cudaStream_t stream) {
   return split > 1 ? launch_swap_form<kRowsA, true>(dev, split, b, m, k, n, map_a, map_b, C, overwrite,
-                                                    bt, stream, launches)
-                   : launch_swap_form<kRowsA, false>(dev, 1, b, m, k, n, map_a, map_b, C, overwrite, bt,
-                                                     stream, launches);
+                                                    bt, stream)
+                   : launch_swap_form<kRowsA, false>(dev, ws_split, b, m, k, n, map_a, map_b, C,
+                                                     overwrite, bt, stream);
 }
 
 }  // namespace
 
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m, int64_t k,
-                        int64_t n, const uint16_t* A, const uint16_t* B, float* C, float*,
+                        int64_t n, const uint16_t* A, const uint16_t* B, float* C, float* workspace,
                         cudaStream_t stream, uint64_t* launches, bool overwrite, bool bt) {
+  // With k slices through the workspace the kernels write partial[slice][b][m][n] there (plain
+  // stores) and the reduce launch below adds the slices and C.
+  const bool sliced = plan.ws_split > 1;
+  if (sliced && !workspace) return cudaErrorInvalidValue;
+  float* out = sliced ? workspace : C;
+  const bool out_overwrite = sliced ? true : overwrite;
   CUtensorMap map_a, map_b, map_c;
-  cudaError_t e = get_maps(MapKey{A, B, C, b, m, k, n, bt}, &map_a, &map_b, &map_c);
+  cudaError_t e = get_maps(MapKey{A, B, out, b, m, k, n, bt, sliced ? plan.ws_split * b : b}, &map_a,
+                           &map_b, &map_c);
   if (e != cudaSuccess) return e;
   const int code = plan.form * 1000 + plan.tile_n;
+  const int wss = plan.ws_split;
   switch (code) {
-    case 3016: return launch_swap<16>(dev, plan.split_k, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
-    case 3032: return launch_swap<32>(dev, plan.split_k, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
-    case 3048: return launch_swap<48>(dev, plan.split_k, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
-    case 3064: return launch_swap<64>(dev, plan.split_k, b, m, k, n, map_a, map_b, C, overwrite, bt, stream, launches);
-    case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, bt, stream); break;
-    case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, bt, stream); break;
-    case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, bt, stream); break;
-    case 2128: e = launch_gemm<true, 128>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, bt, stream); break;
-    case 2256: e = launch_gemm<true, 256>(dev, b, m, k, n, map_a, map_b, map_c, C, plan.halves, overwrite, bt, stream); break;
+    case 3016: e = launch_swap<16>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, stream); break;
+    case 3032: e = launch_swap<32>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, stream); break;
+    case 3048: e = launch_swap<48>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, stream); break;
+    case 3064: e = launch_swap<64>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, stream); break;
+    case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, stream); break;
+    case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, stream); break;
+    case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, stream); break;
+    case 2128: e = launch_gemm<true, 128>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, stream); break;
+    case 2256: e = launch_gemm<true, 256>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, stream); break;
     default: return cudaErrorInvalidValue;
   }
-  if (e == cudaSuccess) ++*launches;
-  return e;
+  if (e != cudaSuccess) return e;
+  ++*launches;
+  if (sliced) {
+    e = skinny_reduce_launch(workspace, C, b, (int)m, n, m * n, plan.ws_split, stream, overwrite);
+    if (e != cudaSuccess) return e;
+    ++*launches;
+  }
+  return cudaSuccess;
 }
 
 }  // namespace morello

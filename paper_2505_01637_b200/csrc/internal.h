@@ -89,6 +89,8 @@ struct GemmPlan {
   size_t workspace_bytes;
   bool halves;   // tiles of a sparse last wave may be cut into column halves
   int split_k;   // operand-swapped kernel only: k slices per strip, added inside a cluster (1, 2, 4, 8)
+  int ws_split;  // > 1: k slices whose sums go to partial[slice][b][m][n] in the workspace and are
+                 // added, slice by slice and then to C, by the reduce kernel
 };
 
 bool gemm_shape_supported(int64_t b, int64_t m, int64_t k, int64_t n, const void* A,

@@ -235,6 +235,30 @@ reduce_kernel(const float* __restrict__ partial, float* __restrict__ C, int64_t 
   *c = overwrite ? sum : *c + sum;
 }
 
+// The same sums, four neighbouring outputs per thread (shapes whose batch sizes and pointers
+// keep every group of four inside one batch and 16-byte aligned).
+__global__ void __launch_bounds__(256)
+reduce4_kernel(const float4* __restrict__ partial, float* __restrict__ C, int64_t total4,
+               int64_t mn, int64_t c_batch, int split_k, int overwrite) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  pdl_wait();
+  pdl_release();
+  if (idx >= total4) return;
+  float4 sum = partial[idx];
+  for (int s = 1; s < split_k; ++s) {
+    const float4 v = partial[(int64_t)s * total4 + idx];
+    sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+  }
+  const int64_t e = idx * 4;
+  const int64_t bb = e / mn;
+  float4* c = reinterpret_cast<float4*>(C + bb * c_batch + (e - bb * mn));
+  if (!overwrite) {
+    const float4 v = *c;
+    sum.x = v.x + sum.x; sum.y = v.y + sum.y; sum.z = v.z + sum.z; sum.w = v.w + sum.w;
+  }
+  *c = sum;
+}
+
 // Launch with programmatic stream serialisation (see pdl_wait above).
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, int threads, size_t smem,
@@ -429,6 +453,14 @@ cudaError_t colmajor_fallback_launch(int64_t b, int64_t m, int64_t k, int64_t n,
 cudaError_t skinny_reduce_launch(const float* partial, float* C, int64_t b, int m, int64_t n,
                                  int64_t c_batch, int split_k, cudaStream_t stream, bool overwrite) {
   const int64_t total = b * m * n;
+  const int64_t mn = (int64_t)m * n;
+  if (mn % 4 == 0 && c_batch % 4 == 0 && reinterpret_cast<uintptr_t>(partial) % 16 == 0 &&
+      reinterpret_cast<uintptr_t>(C) % 16 == 0) {
+    const int64_t total4 = total / 4;
+    return launch_pdl(reduce4_kernel, dim3((unsigned)((total4 + 255) / 256), 1, 1), 256, 0, stream,
+                      reinterpret_cast<const float4*>(partial), C, total4, mn, c_batch, split_k,
+                      overwrite ? 1 : 0);
+  }
   const int64_t blocks = (total + 255) / 256;
   return launch_pdl(reduce_kernel, dim3((unsigned)blocks, 1, 1), 256, 0, stream, partial, C, total,
                     (int64_t)m * n, c_batch, split_k, overwrite ? 1 : 0);

@@ -212,3 +212,68 @@ def test_swap_form_refuses_more_than_64_rows():
     with pytest.raises(mb.MorelloError) as e:
         mb.morello_matmul_accum_forced(TC, SWAP, b, m, k, n, dA, dB, dC)
     assert e.value.status == mb.MORELLO_ERR_UNSUPPORTED_PATH
+
+
+# ------------------------------------------------ k slices through the workspace (few tiles, long k)
+WS = 512   # knob field: number of k slices whose sums go through the workspace
+
+
+@pytest.mark.parametrize("slices", [2, 3, 8])
+@pytest.mark.parametrize("shape,form", [
+    ((1, 128, 2048, 256), 64 + 1),     # one tile of a lone CTA
+    ((1, 300, 1000, 520), 64 + 2),     # pair tiles, ragged m, k and n
+    ((2, 129, 520, 200), 16 + 1),      # 64-column tiles, batches
+    ((1, 256, 4096, 512), 32 + 2),
+    ((1, 64, 2048, 384), SWAP + 16),   # operand-swapped, 64 rows
+    ((2, 5, 1000, 136), SWAP + 16),    # operand-swapped, ragged, batches
+    ((1, 40, 520, 264), SWAP + 16),
+])
+def test_k_slices_through_the_workspace(shape, form, slices):
+    b, m, k, n = shape
+    knob = form + WS * slices
+    A, B, C = w.make(b, m, k, n, seed=sum(shape) + slices, ab="int4", c="normal")
+    got = check_full(A, B, C, integer=True, path=TC, split_k=knob, what="%d slices %s" % (slices, shape))
+    assert_bit_exact(gpu_run(A, B, C, path=TC, split_k=form + WS), got, "slices vs whole k")
+    A, B, C = w.make(b, m, k, n, seed=sum(shape) + slices + 1, ab="normal_rsqrtk", c="normal")
+    first = check_full(A, B, C, integer=False, path=TC, split_k=knob)
+    assert np.array_equal(bits(gpu_run(A, B, C, path=TC, split_k=knob)), bits(first))
+
+
+@pytest.mark.parametrize("shape", [
+    (1, 64, 16384, 2048),    # 16 strips of 64 rows: no cluster, slices through the workspace
+    (1, 128, 16384, 2048),   # one row of tiles
+    (1, 512, 8192, 1024),    # a few pair tiles
+    (1, 8, 8192, 8192),      # 64 strips
+])
+def test_few_tiles_and_a_long_k_by_shape(shape):
+    b, m, k, n = shape
+    assert mb.morello_workspace_bytes(b, m, k, n) >= 2 * b * m * n * 4
+    A, B, C = w.make(b, m, k, n, seed=sum(shape), ab="int4", c="normal")
+    got = check_full(A, B, C, integer=True, what="by shape %s" % (shape,))
+    assert np.array_equal(bits(gpu_run(A, B, C)), bits(got))
+    A, B, C = w.make(b, m, k, n, seed=sum(shape) + 1, ab="normal_rsqrtk", c="normal")
+    check_full(A, B, C, integer=False, what="by shape %s random" % (shape,))
+
+
+def test_k_slices_with_matmul_and_a_caller_workspace():
+    from gpu_util import to_dev
+    import torch
+    b, m, k, n = 1, 128, 4096, 512
+    A, B, C = w.make(b, m, k, n, seed=5, ab="int4", c="normal")
+    knob = 16 + 1 + WS * 4
+    need = mb.morello_workspace_bytes_forced(TC, knob, b, m, k, n)
+    assert need == 4 * b * m * n * 4
+    want = oracle.matmul_accum(b, m, k, n, A, B, C)
+    dA, dB, dC = to_dev(A, B, C)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    mb.morello_matmul_accum_forced(TC, knob, b, m, k, n, dA, dB, dC, ws.data_ptr(), need)
+    torch.cuda.synchronize()
+    assert_bit_exact(dC.cpu().numpy(), want, "caller workspace")
+    with pytest.raises(mb.MorelloError) as e:
+        mb.morello_matmul_accum_forced(TC, knob, b, m, k, n, dA, dB, dC, ws.data_ptr(), need - 16)
+    assert e.value.status == mb.MORELLO_ERR_WORKSPACE
+    # Matmul: C = A x B whatever C held.
+    dC.fill_(float("nan"))
+    mb.morello_matmul_forced(TC, knob, b, m, k, n, dA, dB, dC, 0, 0)
+    torch.cuda.synchronize()
+    assert_bit_exact(dC.cpu().numpy(), oracle.matmul_accum(b, m, k, n, A, B, np.zeros_like(C)), "matmul, slices")
