@@ -118,7 +118,7 @@ int morello_matmul_forced(int path, int split_k,
  * A and C as everywhere else.  With k % 8 == 0, n % 8 == 0 and 16-byte-aligned pointers the
  * tensor-core kernels run it (for them a column-major B is the K-major operand; `tile` is
  * their tile selector as in morello_matmul_accum_forced, 0 = by shape); any other shape
- * runs on a plain one-warp-per-column kernel.  No scratch, no allocation.  Same status
+ * runs on a plain one-warp-per-column kernel.  Scratch as in morello_matmul_accum.  Same status
  * codes, asynchronous on `stream`, deterministic.
  */
 int morello_matmul_accum_colmajor_b(int tile, int64_t b, int64_t m, int64_t k, int64_t n,
@@ -201,13 +201,18 @@ int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n);
  * 16-byte-aligned B; it raises the split as needed to keep the part of A a block
  * stages within 32 KiB: 16384 / m rows of k per block, m rounded up to 1, 2 or 4; up to
  * 8 slices are added inside a thread-block cluster, without scratch), 3 = the same kernel
- * with the slices always added by the reduce kernel from scratch.  On the tcgen05 path, which never
- * splits k, the argument instead selects the tile: (value % 16) is the form -- 0 = by
+ * with the slices always added by the reduce kernel from scratch.  On the tcgen05 path the
+ * argument instead selects the tile: (value % 16) is the form -- 0 = by
  * shape, 1 = one CTA per 128-row tile, 2 = a pair of CTAs per 256-row tile
  * (cta_group::2), 3 = the operand-swapped kernel for at most 64 rows (with it the next
  * field is the number of k slices added inside a cluster instead: 0 = by shape, 1, 2, 4, 8) -- ((value / 16) % 16) is the tile's column count / 64 -- 0 = by
- * shape, 1, 2 or 4 (64 columns only with form 1) -- and adding 256 keeps the tiles of a
- * sparse last wave whole instead of cutting them into column halves.  Returns MORELLO_ERR_UNSUPPORTED_PATH, and
+ * shape, 1, 2 or 4 (64 columns only with form 1) -- adding 256 keeps the tiles of a
+ * sparse last wave whole instead of cutting them into column halves, and ((value / 512) % 16)
+ * is the number of k slices whose partial sums go through the workspace (slices x b x m x n x 4
+ * bytes) and are added in slice order, then to C, by one more launch: 0 = by shape (only
+ * calls whose tiles fill less than half the device and whose k spans at least 32 blocks of 64
+ * are cut), 1 = none, 2 .. 8 (fewer are used if a slice would be empty or the sums would
+ * exceed 64 MiB).  Returns MORELLO_ERR_UNSUPPORTED_PATH, and
  * enqueues nothing, when the path cannot run the shape (the tcgen05 path needs
  * k % 8 == 0, n % 8 == 0 and 16-byte-aligned A, B, C) or the value names no tile.
  * workspace may be NULL with workspace_bytes 0 to use the library's own per-device

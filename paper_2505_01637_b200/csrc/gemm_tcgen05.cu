@@ -938,7 +938,8 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   const int64_t max_units = kPair ? pair_units(dev.sms) : dev.sms;
   // The last wave of a compute-bound problem: when its tiles would occupy at most half the
   // units, each is cut into two column halves so that twice as many units share the wave.
-  // (k is never cut: a second addition into C would make the bits depend on arrival order.)
+  // (Its k is not cut: a second addition into C would make the bits depend on arrival order,
+  // and a trip through the workspace costs more than it saves here.)
   const int64_t tail = p.tiles % max_units;
   if (halves && (S::kColsB / 2) % 64 == 0 && p.tiles > max_units && tail > 0 && 2 * tail <= max_units) {
     p.whole = p.tiles - tail;
