@@ -189,7 +189,11 @@ size_t morello_noalloc_scratch_limit(void);
 /* The path the selector picks for this shape with 16-byte-aligned operands:
  * MORELLO_PATH_SKINNY or MORELLO_PATH_TCGEN05 (-1 for an invalid shape).  A single row
  * (the GEMV) goes to the FP32-FMA kernels; from 2 rows on the tcgen05 kernels run whenever they can
- * address the shape (k % 8 == 0, n % 8 == 0).  (Nothing in the choice depends on the device;
+ * address the shape (k % 8 == 0, n % 8 == 0); other extents with more than 8 rows reach them
+ * through zero-padded copies of the operands in the workspace whenever that is estimated to
+ * cost less than streaming B once per 16 rows on the FMA kernels (also reported as
+ * MORELLO_PATH_TCGEN05; forcing that path means the direct kernels and refuses such
+ * shapes).  (Nothing in the choice depends on the device;
  * 148 SMs are assumed when no device is usable). */
 int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n);
 

@@ -106,6 +106,34 @@ int select_path(int sms, int64_t b, int64_t m, int64_t k, int64_t n, const void*
   return MORELLO_PATH_TCGEN05;
 }
 
+// Extents the TMA engine cannot address (k % 8 != 0 or n % 8 != 0): the FMA kernels take the
+// rows in chunks of 16 and stream B once per chunk, the padded-copy route pays one pass over A
+// and B, one over C and a handful of launches and then runs at tensor-core speed.  Measured
+// (us per call, FMA kernels / padded copies): 512 x 1000 x 1001: 723 / 16.5, 2048 x 2047 x
+// 2049: 9,380 / 48.6, 4096 x 4095 x 4097: 54,352 / 189, 16 x 2048 x 16383: 258 / 48.8, 64 x
+// 1001 x 1001: 91 / 18.5; 17 x 100 x 100 (two chunks): 10.9 on the FMA kernels.
+// Estimated cost of both, in microseconds; pointers that are merely misaligned keep the FMA
+// route (the workspace a shape may need must not depend on them).
+bool staged_wins(int64_t b, int64_t m, int64_t k, int64_t n) {
+  if ((k % 8 == 0 && n % 8 == 0) || m <= 8) return false;
+  const int64_t limit = (1ll << 31) - 8;   // tensor-map extents are 32-bit
+  if (b >= limit || m >= limit || k >= limit || n >= limit) return false;
+  const double bytes_a = 2.0 * b * m * k, bytes_b = 2.0 * b * k * n, bytes_c = 4.0 * b * m * n;
+  const double chunks = (double)((m + 15) / 16);
+  const double fma = chunks * (5.0 + bytes_b * 1.33e-6);
+  const double staged = 14.0 + (2.0 * (bytes_a + bytes_b) + 3.0 * bytes_c) / 5e6 +
+                        2.0 * b * m * k * n / 1e9;
+  return staged < fma;
+}
+
+// Bytes of the padded-copy route's workspace when every operand is staged, its own tensor-core
+// call included.
+size_t staged_workspace(int sms, int64_t b, int64_t m, int64_t k, int64_t n) {
+  const void* odd = reinterpret_cast<const void*>(uintptr_t(4100));   // 4-byte aligned only
+  const PadPlan pp = pad_plan(b, m, k, n, odd, odd, odd);
+  return pp.bytes_a + pp.bytes_b + pp.bytes_c + gemm_plan(sms, b, m, pp.k8, pp.n8, 0).workspace_bytes;
+}
+
 // The knob of the forced entry point on the skinny path: knob % 1024 is the split of the k
 // range (0 = automatic), knob / 1024 picks the kernel (0 = by shape, 1 = the register-
 // streaming kernel, 2 = the TMA-ring GEMV kernel, which needs m <= 4, n % 8 == 0 and a
@@ -178,6 +206,7 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
   }
 
   bool bt_fallback = false;
+  bool staged = false;   // through zero-padded copies of the operands (see pad.cu)
   if (b_col_major) {
     // B as [b][n][k]: the tensor-core kernels when the TMA engine can address the operands,
     // else the one-warp-per-column kernel.  The FMA streaming kernels read B by rows only.
@@ -187,7 +216,8 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     path = MORELLO_PATH_TCGEN05;
     bt_fallback = !tc;
   } else if (path == MORELLO_PATH_AUTO) {
-    path = select_path(st->info.sms, b, m, k, n, A, B, C);
+    staged = staged_wins(b, m, k, n);
+    path = staged ? MORELLO_PATH_TCGEN05 : select_path(st->info.sms, b, m, k, n, A, B, C);
   } else if (path == MORELLO_PATH_TCGEN05) {
     if (!gemm_shape_supported(b, m, k, n, A, B, C)) return MORELLO_ERR_UNSUPPORTED_PATH;
   } else if (path != MORELLO_PATH_SKINNY) {
@@ -201,7 +231,15 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     which = skinny_kernel_for(split_k, b, m, k, n, B);
     if (which < 0) return MORELLO_ERR_UNSUPPORTED_PATH;
   }
-  const size_t need = bt_fallback ? 0 : workspace_for(sms, path, split_k, b, m, k, n, B);
+  PadPlan pad{};
+  GemmPlan pad_gemm{};
+  if (staged) {
+    pad = pad_plan(b, m, k, n, A, B, C);
+    pad_gemm = gemm_plan(sms, b, m, pad.k8, pad.n8, 0);
+    if (!pad_gemm.supported) return MORELLO_ERR_UNSUPPORTED_PATH;
+  }
+  const size_t need = staged ? pad.bytes_a + pad.bytes_b + pad.bytes_c + pad_gemm.workspace_bytes
+                      : bt_fallback ? 0 : workspace_for(sms, path, split_k, b, m, k, n, B);
   float* ws = static_cast<float*>(workspace);
   if (need > 0) {
     if (own_scratch) {
@@ -229,7 +267,23 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   uint64_t launches = 0;
   cudaError_t e = cudaSuccess;
-  if (bt_fallback) {
+  if (staged) {
+    char* base = reinterpret_cast<char*>(ws);
+    uint16_t* a_pad = reinterpret_cast<uint16_t*>(base);
+    uint16_t* b_pad = reinterpret_cast<uint16_t*>(base + pad.bytes_a);
+    float* c_pad = reinterpret_cast<float*>(base + pad.bytes_a + pad.bytes_b);
+    float* inner_ws = reinterpret_cast<float*>(base + pad.bytes_a + pad.bytes_b + pad.bytes_c);
+    e = pad_operands_launch(pad, b, m, k, n, static_cast<const uint16_t*>(A),
+                            static_cast<const uint16_t*>(B), a_pad, b_pad, s, &launches);
+    if (e == cudaSuccess)
+      e = gemm_launch(st->info, pad_gemm, b, m, pad.k8, pad.n8,
+                      pad.stage_a ? a_pad : static_cast<const uint16_t*>(A),
+                      pad.stage_b ? b_pad : static_cast<const uint16_t*>(B),
+                      pad.stage_c ? c_pad : C, pad_gemm.workspace_bytes ? inner_ws : nullptr, s,
+                      &launches, pad.stage_c ? true : overwrite);
+    if (e == cudaSuccess && pad.stage_c)
+      e = unpad_add_launch(pad, b, m, n, c_pad, C, overwrite, s, &launches);
+  } else if (bt_fallback) {
     e = colmajor_fallback_launch(b, m, k, n, static_cast<const uint16_t*>(A),
                                  static_cast<const uint16_t*>(B), C, overwrite, s, &launches);
   } else if (path == MORELLO_PATH_TCGEN05) {
@@ -291,6 +345,8 @@ size_t morello_workspace_bytes_forced(int path, int split_k, int64_t b, int64_t 
     std::lock_guard<std::mutex> lock(g_mutex);
     if (device_state(&st) != MORELLO_OK) return 0;
   }
+  if (path == MORELLO_PATH_AUTO && staged_wins(b, m, k, n))
+    return staged_workspace(st->info.sms, b, m, k, n);
   if (path == MORELLO_PATH_AUTO) path = select_path(st->info.sms, b, m, k, n, fake, fake, fake);
   if (path == MORELLO_PATH_TCGEN05 && !gemm_shape_supported(b, m, k, n, fake, fake, fake)) return 0;
   if (path == MORELLO_PATH_SKINNY && skinny_kernel_for(split_k, b, m, k, n, fake) < 0) return 0;
@@ -435,6 +491,7 @@ int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n) {
     std::lock_guard<std::mutex> lock(g_mutex);
     if (device_state(&st) == MORELLO_OK) sms = st->info.sms;
   }
+  if (!empty && staged_wins(b, m, k, n)) return MORELLO_PATH_TCGEN05;   // through padded copies
   return select_path(sms, b, m, k, n, fake, fake, fake);
 }
 

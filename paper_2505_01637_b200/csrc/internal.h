@@ -81,6 +81,22 @@ cudaError_t f32_split_launch(int64_t b, int64_t m, int64_t k, int64_t n, const f
                              void* split, uint16_t** A6, uint16_t** B6, cudaStream_t stream,
                              uint64_t* launches);
 
+// ---- zero-padded copies of operands the TMA engine cannot address --------------
+struct PadPlan {
+  int64_t k8, n8;                    // k and n rounded up to multiples of 8
+  bool stage_a, stage_b, stage_c;    // which operands go through a padded copy
+  size_t bytes_a, bytes_b, bytes_c;  // their sizes in the workspace (multiples of 256)
+};
+// Which operands need a copy for these extents and pointers.
+PadPlan pad_plan(int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const void* B,
+                 const void* C);
+cudaError_t pad_operands_launch(const PadPlan& p, int64_t b, int64_t m, int64_t k, int64_t n,
+                                const uint16_t* A, const uint16_t* B, uint16_t* A_pad,
+                                uint16_t* B_pad, cudaStream_t stream, uint64_t* launches);
+// C (+)= the first n columns of C_pad[b][m][n8].
+cudaError_t unpad_add_launch(const PadPlan& p, int64_t b, int64_t m, int64_t n, const float* C_pad,
+                             float* C, bool overwrite, cudaStream_t stream, uint64_t* launches);
+
 // ---- tcgen05 path ------------------------------------------------------------
 struct GemmPlan {
   bool supported;

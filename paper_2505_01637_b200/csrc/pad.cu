@@ -1,0 +1,102 @@
+// Shapes the TMA engine cannot address (k % 8 != 0 or n % 8 != 0), with enough rows that the
+// FP32-FMA kernels would stream B many times over: the operands are copied once into
+// zero-padded, 16-byte-aligned buffers in the workspace,
+//     A'[b][m][k8]  (k8 = k rounded up to 8; the added columns are zero),
+//     B'[b][k8][n8] (n8 = n rounded up to 8; the added rows and columns are zero),
+// the tensor-core kernels compute MatmulAccum(b, m, k8, n8) on them -- the zero padding adds
+// exact zeros to every sum -- and, when C's rows cannot be addressed either, the product goes
+// to C'[b][m][n8] first and one elementwise launch adds (or, for Matmul, copies) its first n
+// columns to C.  C is still added exactly once, last, to the complete sum.
+#include "internal.h"
+
+namespace morello {
+namespace {
+
+// dst[bb][r][c] = src[bb][r][c] inside the source extents, else 0; dst is [b][rows_out][cols_out]
+// with cols_out % 8 == 0 and a 16-byte-aligned base.  One thread per 8 output elements.
+__global__ void __launch_bounds__(256)
+pad_bf16_kernel(const uint16_t* __restrict__ src, uint4* __restrict__ dst, int64_t b, int64_t rows_in,
+                int64_t cols_in, int64_t rows_out, int64_t cols_out) {
+  const int64_t groups = cols_out / 8;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= b * rows_out * groups) return;
+  const int64_t g = idx % groups;
+  const int64_t r = (idx / groups) % rows_out;
+  const int64_t bb = idx / (groups * rows_out);
+  uint32_t w[4] = {0u, 0u, 0u, 0u};
+  if (r < rows_in) {
+    const uint16_t* row = src + (bb * rows_in + r) * cols_in;
+    const int64_t c0 = g * 8;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const uint32_t v = (c0 + e < cols_in) ? (uint32_t)row[c0 + e] : 0u;
+      w[e >> 1] |= v << ((e & 1) * 16);
+    }
+  }
+  dst[idx] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// C[bb][i][j] = (overwrite ? 0 : C[bb][i][j]) + P[bb][i][j] for j < n; P is [b][m][n8].
+__global__ void __launch_bounds__(256)
+unpad_add_kernel(const float* __restrict__ P, float* __restrict__ C, int64_t rows, int64_t n,
+                 int64_t n8, int overwrite) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= rows * n) return;
+  const int64_t r = idx / n, j = idx - r * n;
+  const float sum = P[r * n8 + j];
+  C[idx] = overwrite ? sum : C[idx] + sum;
+}
+
+size_t round256(size_t x) { return (x + 255) / 256 * 256; }
+
+}  // namespace
+
+PadPlan pad_plan(int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const void* B,
+                 const void* C) {
+  PadPlan p{};
+  p.k8 = (k + 7) / 8 * 8;
+  p.n8 = (n + 7) / 8 * 8;
+  const bool k_odd = (k % 8) != 0, n_odd = (n % 8) != 0;
+  p.stage_a = k_odd || reinterpret_cast<uintptr_t>(A) % 16 != 0;
+  p.stage_b = k_odd || n_odd || reinterpret_cast<uintptr_t>(B) % 16 != 0;
+  p.stage_c = n_odd || reinterpret_cast<uintptr_t>(C) % 16 != 0;
+  p.bytes_a = p.stage_a ? round256((size_t)b * m * p.k8 * 2) : 0;
+  p.bytes_b = p.stage_b ? round256((size_t)b * p.k8 * p.n8 * 2) : 0;
+  p.bytes_c = p.stage_c ? round256((size_t)b * m * p.n8 * 4) : 0;
+  return p;
+}
+
+cudaError_t pad_operands_launch(const PadPlan& p, int64_t b, int64_t m, int64_t k, int64_t n,
+                                const uint16_t* A, const uint16_t* B, uint16_t* A_pad,
+                                uint16_t* B_pad, cudaStream_t stream, uint64_t* launches) {
+  if (p.stage_a) {
+    const int64_t threads = b * m * (p.k8 / 8);
+    pad_bf16_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(
+        A, reinterpret_cast<uint4*>(A_pad), b, m, k, m, p.k8);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    ++*launches;
+  }
+  if (p.stage_b) {
+    const int64_t threads = b * p.k8 * (p.n8 / 8);
+    pad_bf16_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(
+        B, reinterpret_cast<uint4*>(B_pad), b, k, n, p.k8, p.n8);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    ++*launches;
+  }
+  return cudaSuccess;
+}
+
+cudaError_t unpad_add_launch(const PadPlan& p, int64_t b, int64_t m, int64_t n, const float* C_pad,
+                             float* C, bool overwrite, cudaStream_t stream, uint64_t* launches) {
+  const int64_t total = b * m * n;
+  unpad_add_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(C_pad, C, b * m, n, p.n8,
+                                                                        overwrite ? 1 : 0);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  ++*launches;
+  return cudaSuccess;
+}
+
+}  // namespace morello

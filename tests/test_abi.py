@@ -69,8 +69,10 @@ def test_selector_is_shape_based(mb):
     assert mb.morello_select_path(1, 2, 2048, 16384) == mb.MORELLO_PATH_TCGEN05
     assert mb.morello_select_path(1, 2, 2048, 1024) == mb.MORELLO_PATH_TCGEN05     # few columns: k is cut instead
     assert mb.morello_select_path(1, 16, 4096, 64) == mb.MORELLO_PATH_TCGEN05
-    assert mb.morello_select_path(1, 16, 4096, 60) == mb.MORELLO_PATH_SKINNY        # n % 8 != 0: TMA cannot address it
-    assert mb.morello_select_path(1, 4096, 4096, 4095) == mb.MORELLO_PATH_SKINNY   # n % 8 != 0
+    assert mb.morello_select_path(1, 8, 4096, 60) == mb.MORELLO_PATH_SKINNY         # n % 8 != 0: TMA cannot address it
+    assert mb.morello_select_path(1, 17, 100, 100) == mb.MORELLO_PATH_SKINNY       # ... and too small to be worth copying
+    assert mb.morello_select_path(1, 4096, 4096, 4095) == mb.MORELLO_PATH_TCGEN05  # ... through zero-padded copies
+    assert mb.morello_select_path(1, 512, 1001, 1000) == mb.MORELLO_PATH_TCGEN05   # k % 8 != 0 likewise
     assert mb.morello_select_path(1, 4096, 4096, 4096) == mb.MORELLO_PATH_TCGEN05
     assert mb.morello_select_path(8, 2048, 2048, 16384) == mb.MORELLO_PATH_TCGEN05
     assert mb.morello_select_path(1, 17, 8, 8) == mb.MORELLO_PATH_TCGEN05
