@@ -188,12 +188,15 @@ size_t morello_noalloc_scratch_limit(void);
 
 /* The path the selector picks for this shape with 16-byte-aligned operands:
  * MORELLO_PATH_SKINNY or MORELLO_PATH_TCGEN05 (-1 for an invalid shape).  A single row
- * (the GEMV) goes to the FP32-FMA kernels; from 2 rows on the tcgen05 kernels run whenever they can
- * address the shape (k % 8 == 0, n % 8 == 0); other extents with more than 8 rows reach them
+ * (the GEMV) goes to the FP32-FMA kernels when its 64-column strips fill the device's block
+ * slots about once and k is short (the 1 x 2048 x 16384 case), or when B is small or not
+ * addressable by the TMA engine, and to the operand-swapped tcgen05 kernel otherwise (it
+ * streams long or many-strip B faster); from 2 rows on the tcgen05 kernels run whenever they can
+ * address the shape (k % 8 == 0, n % 8 == 0); other extents with at least 2 rows reach them
  * through zero-padded copies of the operands in the workspace whenever that is estimated to
- * cost less than streaming B once per 16 rows on the FMA kernels (also reported as
+ * cost less than the FMA kernels, which stream B once per 16 rows (also reported as
  * MORELLO_PATH_TCGEN05; forcing that path means the direct kernels and refuses such
- * shapes).  (Nothing in the choice depends on the device;
+ * shapes).  (The single-row choice looks at the device's SM count;
  * 148 SMs are assumed when no device is usable). */
 int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n);
 

@@ -100,9 +100,26 @@ int validate(int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const vo
 constexpr int kFmaMaxRows = 1;
 int select_path(int sms, int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const void* B,
                 const void* C) {
-  (void)sms;
-  if (m <= kFmaMaxRows) return MORELLO_PATH_SKINNY;
   if (!gemm_shape_supported(b, m, k, n, A, B, C)) return MORELLO_PATH_SKINNY;
+  if (m <= kFmaMaxRows) {
+    // The single row.  The FMA GEMV kernel is at its best when its 64-column strips (times its
+    // k slices) fill the two block slots per SM exactly once and k is short; elsewhere the
+    // operand-swapped tensor kernel streams B faster (128-column strips, deeper ring).
+    // Measured, us per call, FMA GEMV / operand-swapped, k x n: 2048 x 8192: 8.2 / 9.2; 2048 x
+    // 16384: 11.1 / 11.5; 4096 x 8192: 12.3 / 13.8; 8192 x 8192: 22.7 / 23.3; but 2048 x 12288
+    // (384 blocks): 13.9 / 9.9; 2048 x 20480: 19.1 / 14.0; 4096 x 32000: 45.9 / 40.0; 4096 x
+    // 16384: 21.6 / 20.8; 8192 x 16384: 41.3 / 39.3; 4096 x 65536: 87.2 / 81.3.
+    // (Below 16 MB of B both finish within a launch latency or two; the FMA kernels are the
+    // lighter launch: 2048 x 2048: 4.7 / 5.4.)
+    if (b > 65535 || b * k * n < (1ll << 23) || !stream_shape_supported(b, 1, k, n, B))
+      return MORELLO_PATH_SKINNY;
+    const StreamPlan pl = stream_plan(sms, b, 1, k, n, 0);
+    if (!pl.supported) return MORELLO_PATH_TCGEN05;
+    const int64_t blocks = b * pl.strips * pl.split_k, slots = 2ll * sms;
+    const bool one_full_wave = blocks <= slots && blocks * 5 >= slots * 4;
+    if (one_full_wave && (k <= 2048 || (b * pl.strips <= 128 && k <= 16384))) return MORELLO_PATH_SKINNY;
+    return MORELLO_PATH_TCGEN05;
+  }
   return MORELLO_PATH_TCGEN05;
 }
 
@@ -113,16 +130,26 @@ int select_path(int sms, int64_t b, int64_t m, int64_t k, int64_t n, const void*
 // 2049: 9,380 / 48.6, 4096 x 4095 x 4097: 54,352 / 189, 16 x 2048 x 16383: 258 / 48.8, 64 x
 // 1001 x 1001: 91 / 18.5; 17 x 100 x 100 (two chunks): 10.9 on the FMA kernels.
 // Estimated cost of both, in microseconds; pointers that are merely misaligned keep the FMA
-// route (the workspace a shape may need must not depend on them).
+// route (the workspace a shape may need must not depend on them).  2 to 8 rows, 2048 x 16383,
+// FMA / copies: 2 rows 35.7 / 48, 4 rows 86 / 48, 8 rows 119 / 48.
 bool staged_wins(int64_t b, int64_t m, int64_t k, int64_t n) {
-  if ((k % 8 == 0 && n % 8 == 0) || m <= 8) return false;
+  if ((k % 8 == 0 && n % 8 == 0) || m < 2) return false;
   const int64_t limit = (1ll << 31) - 8;   // tensor-map extents are 32-bit
   if (b >= limit || m >= limit || k >= limit || n >= limit) return false;
   const double bytes_a = 2.0 * b * m * k, bytes_b = 2.0 * b * k * n, bytes_c = 4.0 * b * m * n;
-  const double chunks = (double)((m + 15) / 16);
-  const double fma = chunks * (5.0 + bytes_b * 1.33e-6);
-  const double staged = 14.0 + (2.0 * (bytes_a + bytes_b) + 3.0 * bytes_c) / 5e6 +
-                        2.0 * b * m * k * n / 1e9;
+  // The FMA kernel's cost per MB of B for a chunk of r rows: bound by memory up to a few rows,
+  // then by one FMA per row and element; narrower loads (n % 8, 4, 2 != 0) cost more of both
+  // (measured on 2048 x 16383 / 16382 / 16380, 1 to 8 rows).
+  const int vec = n % 8 == 0 ? 8 : n % 4 == 0 ? 4 : n % 2 == 0 ? 2 : 1;
+  const double base = vec == 8 ? 0.2 : vec == 4 ? 0.3 : vec == 2 ? 0.37 : 0.5;
+  const double per_row = vec == 8 ? 0.083 : vec == 4 ? 0.09 : vec == 2 ? 0.13 : 0.3;
+  const double mb_b = bytes_b / 1e6;
+  const int64_t full_chunks = m / 16, rest = m % 16;
+  double fma = (double)full_chunks * (5.0 + mb_b * std::max(base, 16 * per_row));
+  if (rest) fma += 5.0 + mb_b * std::max(base, (double)rest * per_row);
+  // Copies in and out, then the tensor-core call itself: its FLOPs or its pass over memory.
+  const double staged = 14.0 + (2.0 * (bytes_a + bytes_b) + 3.0 * bytes_c) / 4.4e6 +
+                        std::max(2.0 * b * m * k * n / 1e9, (bytes_a + bytes_b + 2.0 * bytes_c) / 6e6);
   return staged < fma;
 }
 
