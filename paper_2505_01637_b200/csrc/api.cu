@@ -126,23 +126,24 @@ int select_path(int sms, int64_t b, int64_t m, int64_t k, int64_t n, const void*
 // Extents the TMA engine cannot address (k % 8 != 0 or n % 8 != 0): the FMA kernels take the
 // rows in chunks of 16 and stream B once per chunk, the padded-copy route pays one pass over A
 // and B, one over C and a handful of launches and then runs at tensor-core speed.  Measured
-// (us per call, FMA kernels / padded copies): 512 x 1000 x 1001: 723 / 16.5, 2048 x 2047 x
+// (us per call, FMA kernels with narrow loads / padded copies): 512 x 1000 x 1001: 723 / 16.5, 2048 x 2047 x
 // 2049: 9,380 / 48.6, 4096 x 4095 x 4097: 54,352 / 189, 16 x 2048 x 16383: 258 / 48.8, 64 x
 // 1001 x 1001: 91 / 18.5; 17 x 100 x 100 (two chunks): 10.9 on the FMA kernels.
 // Estimated cost of both, in microseconds; pointers that are merely misaligned keep the FMA
-// route (the workspace a shape may need must not depend on them).  2 to 8 rows, 2048 x 16383,
-// FMA / copies: 2 rows 35.7 / 48, 4 rows 86 / 48, 8 rows 119 / 48.
+// route (the workspace a shape may need must not depend on them).
 bool staged_wins(int64_t b, int64_t m, int64_t k, int64_t n) {
   if ((k % 8 == 0 && n % 8 == 0) || m < 2) return false;
   const int64_t limit = (1ll << 31) - 8;   // tensor-map extents are 32-bit
   if (b >= limit || m >= limit || k >= limit || n >= limit) return false;
   const double bytes_a = 2.0 * b * m * k, bytes_b = 2.0 * b * k * n, bytes_c = 4.0 * b * m * n;
   // The FMA kernel's cost per MB of B for a chunk of r rows: bound by memory up to a few rows,
-  // then by one FMA per row and element; narrower loads (n % 8, 4, 2 != 0) cost more of both
-  // (measured on 2048 x 16383 / 16382 / 16380, 1 to 8 rows).
+  // then by one FMA per row and element.  Its flat form reads unaligned rows in aligned
+  // 16-byte granules (measured on 2048 x 16383, us per call: 1 row 16.6, 2: 19.6, 4: 24.6,
+  // 8: 37.1, 16: 79.1); tiny shapes fall back to narrow loads, which cost more of both.
+  const bool flat = k >= 64 && n >= 16;
   const int vec = n % 8 == 0 ? 8 : n % 4 == 0 ? 4 : n % 2 == 0 ? 2 : 1;
-  const double base = vec == 8 ? 0.2 : vec == 4 ? 0.3 : vec == 2 ? 0.37 : 0.5;
-  const double per_row = vec == 8 ? 0.083 : vec == 4 ? 0.09 : vec == 2 ? 0.13 : 0.3;
+  const double base = flat ? 0.25 : vec == 8 ? 0.2 : vec == 4 ? 0.3 : vec == 2 ? 0.37 : 0.5;
+  const double per_row = flat ? 0.074 : vec == 8 ? 0.083 : vec == 4 ? 0.09 : vec == 2 ? 0.13 : 0.3;
   const double mb_b = bytes_b / 1e6;
   const int64_t full_chunks = m / 16, rest = m % 16;
   double fma = (double)full_chunks * (5.0 + mb_b * std::max(base, 16 * per_row));

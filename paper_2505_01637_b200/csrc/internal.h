@@ -22,6 +22,8 @@ struct DeviceInfo {
 struct SkinnyPlan {
   int m_tile;        // 1, 2, 4, 8 or 16: compile-time row count of the kernel used
   int vec;           // bf16 elements per load: 8, 4, 2 or 1
+  bool flat;         // aligned 16-byte granules with per-row-lane column shifts (B's rows are not
+                     // 16-byte aligned); units then counts one granule more than the block's columns
   int units;         // column units (of `vec` columns) per thread block
   int row_lanes;     // k rows visited per pass of a thread block
   int threads;       // launch width (multiple of 32, >= units * row_lanes)

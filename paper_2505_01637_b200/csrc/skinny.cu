@@ -14,6 +14,19 @@
 // block adds its sums to C itself; with several it writes them to
 // partial[slice][b][m][n] and reduce_kernel adds the slices in slice order and
 // then adds C once.
+//
+// Flat form (FLAT, 16-byte loads only): when n % 8 != 0 or B is not 16-byte aligned, the rows
+// of B start at varying offsets inside their 16-byte granules and the plain form falls back
+// to 8-, 4- or 2-byte loads, several times slower.  Instead every thread loads ALIGNED
+// 16-byte granules: for row p and column block cb, granule ul of the thread block starts d
+// elements before column cb * W + 8 ul, d = the offset of (p, cb * W) inside its granule.
+// d depends only on p mod 8 (8 rows of n elements shift by whole granules), and a thread's
+// rows are 8 | row_lanes apart, so d is a constant of the thread: its 8 accumulators simply
+// belong to columns shifted left by d.  A block carries one granule more than its W / 8
+// (columns W .. W + 7 - d of the shifted windows), the final sum over the row lanes reads
+// lane r's value of column x at index x + d_r, and accumulators of columns outside [0, n)
+// (the neighbouring rows' elements a granule also holds) are never read.  Loads stay inside
+// the 16-byte granules that hold bytes of B.
 #include <algorithm>
 
 #include "internal.h"
@@ -40,6 +53,7 @@ struct SkinnyParams {
   int split_k;
   int k_chunk;
   int overwrite;  // 1: C = sum instead of C += sum
+  int flat_cols;  // flat form: output columns per thread block, 8 * (units - 1)
 };
 
 template <int M_T>
@@ -118,9 +132,10 @@ __device__ __forceinline__ void fma_row(float (&acc)[M_T][VEC], const float* __r
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;"); }
 
-template <int M_T, int VEC, int UNROLL, int THREADS>
+template <int M_T, int VEC, int UNROLL, int THREADS, bool FLAT = false>
 __global__ void __launch_bounds__(THREADS)
 skinny_kernel(const SkinnyParams p) {
+  static_assert(!FLAT || VEC == 8, "the flat form loads whole 16-byte granules");
   extern __shared__ __align__(16) float smem[];
   float* a_s = smem;                                  // [k_chunk][M_T]
   float* red = smem + (size_t)p.k_chunk * M_T;        // [row_lanes][M_T * units * VEC]
@@ -132,7 +147,6 @@ skinny_kernel(const SkinnyParams p) {
   const int s = blockIdx.x / p.col_blocks;
   const int bb = blockIdx.y;
   const int unit = cb * p.units + ul;
-  const bool active = (rl < p.row_lanes) && (unit < p.num_units);
   const int64_t k0 = (int64_t)s * p.k_per_split;
   const int64_t k1 = min(p.k, k0 + p.k_per_split);
   const int R = p.row_lanes;
@@ -145,7 +159,19 @@ skinny_kernel(const SkinnyParams p) {
     for (int j = 0; j < VEC; ++j) acc[i][j] = 0.f;
 
   const uint16_t* a_base = p.A + (int64_t)bb * p.a_batch;
-  const uint16_t* bp = p.B + (int64_t)bb * p.b_batch + (int64_t)unit * VEC + (k0 + rl) * p.n;
+  // Element index (address / 2) of (row 0 of the batch, first column of this column block).
+  const uint64_t flat_e0 = (reinterpret_cast<uint64_t>(p.B) >> 1) + (uint64_t)bb * p.b_batch +
+                           (uint64_t)cb * p.flat_cols;
+  // First column of the thread's accumulators: plain form unit * VEC; flat form the column
+  // block's first column, back by this row lane's offset d, plus 8 ul.
+  int64_t col_off = (int64_t)unit * VEC;
+  bool active = (rl < p.row_lanes) && (unit < p.num_units);
+  if constexpr (FLAT) {
+    const int d = (int)((flat_e0 + (uint64_t)(k0 + rl) * p.n) & 7u);
+    col_off = (int64_t)cb * p.flat_cols - d + 8 * ul;
+    active = (rl < p.row_lanes) && col_off < p.n;
+  }
+  const uint16_t* bp = p.B + (int64_t)bb * p.b_batch + col_off + (k0 + rl) * p.n;
 
   // The first group of B rows is requested before A is staged, so that the staging
   // latency hides under the first HBM round trip.  Nothing is touched before pdl_wait().
@@ -189,7 +215,7 @@ skinny_kernel(const SkinnyParams p) {
           if (q + u * R < kcl) fma_row<M_T, VEC>(acc, a_s + (q + u * R) * M_T, v[u]);
       }
       // bp now points UNROLL*R-aligned past the chunk; rebase to the next chunk's first row.
-      bp = p.B + (int64_t)bb * p.b_batch + (int64_t)unit * VEC + (kc0 + kcl + rl) * p.n;
+      bp = p.B + (int64_t)bb * p.b_batch + col_off + (kc0 + kcl + rl) * p.n;
     }
   }
 
@@ -203,6 +229,29 @@ skinny_kernel(const SkinnyParams p) {
       for (int j = 0; j < VEC; ++j) dst[i * p.units * VEC + j] = acc[i][j];
   }
   __syncthreads();
+  if constexpr (FLAT) {
+    // Row lane r holds column x of this block at index x + d_r of its row of sums.
+    const int cols = p.flat_cols;
+    const int pitch = p.units * VEC;
+    for (int o = t; o < M_T * cols; o += blockDim.x) {
+      const int i = o / cols, x = o - i * cols;
+      const int64_t col = (int64_t)cb * cols + x;
+      if (i >= p.m || col >= p.n) continue;
+      float sum = 0.f;
+      for (int r = 0; r < R; ++r) {
+        const int d = (int)((flat_e0 + (uint64_t)(k0 + r) * p.n) & 7u);
+        const float v = red[(size_t)r * W + i * pitch + x + d];
+        sum = r == 0 ? v : sum + v;
+      }
+      if (p.split_k == 1) {
+        float* c = p.C + (int64_t)bb * p.c_batch + (int64_t)i * p.n + col;
+        *c = p.overwrite ? sum : *c + sum;
+      } else {
+        p.partial[(int64_t)s * p.partial_split_stride + ((int64_t)bb * p.m + i) * p.n + col] = sum;
+      }
+    }
+    return;
+  }
   const int cols_here = p.units * VEC;
   const int64_t col_base = (int64_t)cb * cols_here;
   for (int o = t; o < W; o += blockDim.x) {
@@ -290,8 +339,22 @@ cudaError_t launch_one(const SkinnyPlan& plan, const SkinnyParams& prm, int64_t 
 }
 
 template <int M_T>
+cudaError_t launch_flat(const SkinnyPlan& plan, const SkinnyParams& prm, int64_t b,
+                        cudaStream_t stream) {
+  auto kern = skinny_kernel<M_T, 8, Tuning<M_T>::kUnroll, Tuning<M_T>::kThreads, true>;
+  if (plan.smem_bytes > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)plan.smem_bytes);
+    if (e != cudaSuccess) return e;
+  }
+  dim3 grid((unsigned)(plan.col_blocks * plan.split_k), (unsigned)b, 1);
+  return launch_pdl(kern, grid, plan.threads, plan.smem_bytes, stream, prm);
+}
+
+template <int M_T>
 cudaError_t launch_vec(const SkinnyPlan& plan, const SkinnyParams& prm, int64_t b,
                        cudaStream_t stream) {
+  if (plan.flat) return launch_flat<M_T>(plan, prm, b, stream);
   switch (plan.vec) {
     case 8: return launch_one<M_T, 8>(plan, prm, b, stream);
     case 4: return launch_one<M_T, 4>(plan, prm, b, stream);
@@ -319,12 +382,16 @@ int skinny_vec(int64_t n, const void* B) {
   return 1;
 }
 
-SkinnyPlan skinny_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int vec, int split_k) {
+namespace {
+
+SkinnyPlan plan_impl(int sms, int64_t b, int m, int64_t k, int64_t n, int vec, int split_k, bool flat) {
   SkinnyPlan pl{};
   pl.m_tile = m <= 1 ? 1 : m <= 2 ? 2 : m <= 4 ? 4 : m <= 8 ? 8 : 16;
+  pl.flat = flat;
+  if (flat) vec = 8;
   pl.vec = vec;
   const int max_threads = max_threads_for(pl.m_tile);
-  const int64_t num_units = n / vec;
+  const int64_t num_units = flat ? (n + 7) / 8 : n / vec;
   const int unit_cap = (int)std::min<int64_t>(num_units, 128 / vec);  // <= 256-byte row segments
   // One wave of thread blocks over the SMs when the columns allow it.
   const int64_t per_sm = (b * num_units + sms - 1) / sms;
@@ -336,8 +403,9 @@ SkinnyPlan skinny_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int vec,
     units = (int)((per_sm + waves - 1) / waves);
   }
   units = std::min<int>(units, unit_cap);
-  pl.units = units;
   pl.col_blocks = (int)((num_units + units - 1) / units);
+  if (flat) ++units;   // the granule that holds the shifted windows' last columns
+  pl.units = units;
   const int64_t blocks = b * pl.col_blocks;
   int s = split_k;
   if (s <= 0) {
@@ -364,6 +432,18 @@ SkinnyPlan skinny_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int vec,
   return pl;
 }
 
+}  // namespace
+
+SkinnyPlan skinny_plan(int sms, int64_t b, int m, int64_t k, int64_t n, int vec, int split_k) {
+  // Loads narrower than 16 bytes: the flat form (aligned granules, shifted columns) instead,
+  // once there is a stream of B worth it.  It needs row lanes in multiples of 8.
+  if (vec < 8 && k >= 64 && n >= 16) {
+    const SkinnyPlan flat = plan_impl(sms, b, m, k, n, 8, split_k, true);
+    if (flat.row_lanes % 8 == 0) return flat;
+  }
+  return plan_impl(sms, b, m, k, n, vec, split_k, false);
+}
+
 cudaError_t skinny_launch(const SkinnyPlan& plan, int64_t b, int m, int64_t k, int64_t n,
                           const uint16_t* A, int64_t a_batch, const uint16_t* B, float* C,
                           int64_t c_batch, float* workspace, cudaStream_t stream,
@@ -377,6 +457,7 @@ cudaError_t skinny_launch(const SkinnyPlan& plan, int64_t b, int m, int64_t k, i
   prm.partial_split_stride = b * m * n;
   prm.m = m;
   prm.num_units = (int)(n / plan.vec);
+  prm.flat_cols = plan.flat ? 8 * (plan.units - 1) : 0;
   prm.units = plan.units;
   prm.row_lanes = plan.row_lanes;
   prm.col_blocks = plan.col_blocks;
