@@ -304,6 +304,48 @@ def bench_config(torch, mb, idx, iters, warmup, peaks, windows, path=None, split
     return rec
 
 
+def bench_shape(torch, mb, name, shape, iters, peaks, windows, note):
+    """A shape outside the named configs, through the plain entry point: the selector's other
+    routes (k slices through the workspace, padded copies, the flat FMA form, the single row
+    on the tensor kernel).  Inputs rotate like bench_config's; normal(0, 1/sqrt(k)) values."""
+    b, m, k, n = shape
+    in_bytes = 2 * b * m * k + 2 * b * k * n + 4 * b * m * n
+    sets = max(1, min(ROTATE, int(np.ceil(512 * 2 ** 20 / in_bytes))))
+    dev = []
+    for s_ in range(sets):
+        As, Bs, Cs = w.make(b, m, k, n, 9000 + 10 * s_ + (m + k + n) % 7, "normal_rsqrtk", "zeros")
+        dev.append((torch.from_numpy(As.view(np.int16)).cuda(), torch.from_numpy(Bs.view(np.int16)).cuda(),
+                    torch.from_numpy(Cs).cuda()))
+    ptrs = [(a.data_ptr(), bb.data_ptr(), c.data_ptr()) for (a, bb, c) in dev]
+    stream = torch.cuda.current_stream().cuda_stream
+    call = mb.lib().morello_matmul_accum
+
+    def step(i):
+        pa, pb, pc = ptrs[i % sets]
+        rc = call(b, m, k, n, pa, pb, pc, stream)
+        if rc != 0:
+            raise mb.MorelloError(rc, "bench %s" % name)
+
+    l0 = mb.morello_launch_count()
+    step(0)
+    per_call = mb.morello_launch_count() - l0
+    t0 = time.perf_counter()
+    loops = [time_calls(torch, step, iters, 5 if r == 0 else 3) for r in range(3)]
+    windows.append((t0, time.perf_counter()))
+    sec = min(loops) / iters
+    st, detail = mb.morello_read_device_status()
+    if st != 0:
+        raise RuntimeError("device status %d (0x%x) after %s" % (st, detail, name))
+    alg = in_bytes + 4 * b * m * n
+    flops = 2.0 * b * m * k * n
+    return {"name": name, "op": "matmul_accum", "shape": list(shape),
+            "path": "tcgen05" if mb.morello_select_path(b, m, k, n) == 1 else "skinny",
+            "us_per_call": sec * 1e6, "GBps": alg / sec / 1e9, "TFLOPs": flops / sec / 1e12,
+            "iters": iters, "launches_per_call": per_call, "rotating_sets": sets,
+            "frac_hbm_measured": alg / sec / 1e9 / peaks["hbm_gbs"],
+            "frac_tensor_measured_burst": flops / sec / 1e12 / peaks["bf16_tflops"], "note": note}
+
+
 def bench_f32_square(torch, mb, peaks, windows, size=2048, iters=20):
     """The paper's float32 benchmark shape (Section 7: a float32 2048-square matmul) through
     morello_matmul_accum_f32: float32 FLOPs per second, and the bf16 tensor-core FLOPs the
@@ -545,6 +587,12 @@ def run_ours(args):
         extra.append(bench_colmajor(torch, mb, HEADLINE, 300, peaks, windows))
         if 3 in args.configs:
             extra.append(bench_colmajor(torch, mb, 3, 30, peaks, windows))
+        for name, shape, iters, note in (
+                ("route_gemv_long_k", (1, 1, 8192, 16384), 100, "single row on the operand-swapped tensor kernel"),
+                ("route_k_slices", (1, 512, 16384, 2048), 100, "few tiles, long k: k slices through the workspace + reduce launch"),
+                ("route_padded_copies", (1, 2048, 2047, 2049), 50, "k, n not multiples of 8: zero-padded copies, tensor kernels, unpad-add"),
+                ("route_flat_gemv", (1, 1, 2048, 16383), 100, "n odd, one row: FMA kernel reading aligned 16-byte granules")):
+            extra.append(bench_shape(torch, mb, name, shape, iters, peaks, windows, note))
     sampler.stop()
     clocks = sampler.summary(windows)
 
