@@ -428,6 +428,11 @@ def run_case(args):
     mb.lib()
     peaks, _ = load_peaks()
     path = {"auto": None, "skinny": mb.MORELLO_PATH_SKINNY, "tcgen05": mb.MORELLO_PATH_TCGEN05}[args.path]
+    if args.shape:
+        shape = tuple(int(x) for x in args.shape.split(","))
+        rec = bench_shape(torch, mb, "shape", shape, args.steps, peaks, [], "--shape, by the selector")
+        print(json.dumps(rec))
+        return 0
     rec = bench_config(torch, mb, args.case - 1, args.steps, args.warmup, peaks, [], path=path,
                        split_k=args.split)
     rec["case"] = args.case
@@ -656,13 +661,15 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "skinny", "tcgen05"],
                     help="kernel family for --case")
     ap.add_argument("--split", type=int, default=0, help="forced split / form knob for --case")
+    ap.add_argument("--shape", default="",
+                    help="b,m,k,n: time this shape alone through the plain entry point (like --case)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     args.steps = max(args.steps, 1)
     args.configs = [int(x) - 1 for x in args.configs.split(",") if x.strip()]
     if args.impl == "reference":
         return run_reference(args)
-    if args.case:
+    if args.case or args.shape:
         return run_case(args)
     return run_ours(args)
 
