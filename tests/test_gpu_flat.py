@@ -96,3 +96,9 @@ def test_selector_reaches_the_flat_form():
         A, B, C = w.make(b, m, k, n, seed=1, ab="int4", c="int8")
         got = check_full(A, B, C, integer=True, what="auto %s" % (shape,))
         assert_bit_exact(gpu_run(A, B, C, path=SK, split_k=REG), got, "auto vs forced register kernel")
+
+
+def test_flat_form_with_more_batches_than_a_grid_dimension():
+    b, m, k, n = 66000, 1, 64, 17       # two slabs of batches; every slab starts at another offset
+    A, B, C = w.make(b, m, k, n, seed=2, ab="int4", c="int8")
+    check_full(A, B, C, integer=True, path=SK, split_k=REG, what="66000 batches")
