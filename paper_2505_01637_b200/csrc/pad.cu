@@ -8,9 +8,30 @@
 // to C'[b][m][n8] first and one elementwise launch adds (or, for Matmul, copies) its first n
 // columns to C.  C is still added exactly once, last, to the complete sum.
 #include "internal.h"
+#include "sm100.cuh"
 
 namespace morello {
 namespace {
+
+// The copies, the tensor-core call and the unpad-add form a chain of short launches: each is
+// launched with programmatic stream serialisation, waits for its predecessor before it touches
+// global memory and lets its successor's blocks be scheduled right away, so that the launch
+// latencies overlap.  (Every kernel of the chain executes the wait, so "the predecessor has
+// completed" carries through the whole chain.)
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kern)(KArgs...), unsigned blocks, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(blocks, 1, 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
 
 // dst[bb][r][c] = src[bb][r][c] inside the source extents, else 0; dst is [b][rows_out][cols_out]
 // with cols_out % 8 == 0 and a 16-byte-aligned base.  One thread per 8 output elements.
@@ -19,6 +40,8 @@ pad_bf16_kernel(const uint16_t* __restrict__ src, uint4* __restrict__ dst, int64
                 int64_t cols_in, int64_t rows_out, int64_t cols_out) {
   const int64_t groups = cols_out / 8;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  sm100::pdl_wait();
+  sm100::pdl_release();
   if (idx >= b * rows_out * groups) return;
   const int64_t g = idx % groups;
   const int64_t r = (idx / groups) % rows_out;
@@ -41,6 +64,8 @@ __global__ void __launch_bounds__(256)
 unpad_add_kernel(const float* __restrict__ P, float* __restrict__ C, int64_t rows, int64_t n,
                  int64_t n8, int overwrite) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  sm100::pdl_wait();
+  sm100::pdl_release();
   if (idx >= rows * n) return;
   const int64_t r = idx / n, j = idx - r * n;
   const float sum = P[r * n8 + j];
@@ -71,17 +96,15 @@ cudaError_t pad_operands_launch(const PadPlan& p, int64_t b, int64_t m, int64_t 
                                 uint16_t* B_pad, cudaStream_t stream, uint64_t* launches) {
   if (p.stage_a) {
     const int64_t threads = b * m * (p.k8 / 8);
-    pad_bf16_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(
-        A, reinterpret_cast<uint4*>(A_pad), b, m, k, m, p.k8);
-    const cudaError_t e = cudaGetLastError();
+    const cudaError_t e = launch_chained(pad_bf16_kernel, (unsigned)((threads + 255) / 256), stream, A,
+                                         reinterpret_cast<uint4*>(A_pad), b, m, k, m, p.k8);
     if (e != cudaSuccess) return e;
     ++*launches;
   }
   if (p.stage_b) {
     const int64_t threads = b * p.k8 * (p.n8 / 8);
-    pad_bf16_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, stream>>>(
-        B, reinterpret_cast<uint4*>(B_pad), b, k, n, p.k8, p.n8);
-    const cudaError_t e = cudaGetLastError();
+    const cudaError_t e = launch_chained(pad_bf16_kernel, (unsigned)((threads + 255) / 256), stream, B,
+                                         reinterpret_cast<uint4*>(B_pad), b, k, n, p.k8, p.n8);
     if (e != cudaSuccess) return e;
     ++*launches;
   }
@@ -91,9 +114,8 @@ cudaError_t pad_operands_launch(const PadPlan& p, int64_t b, int64_t m, int64_t 
 cudaError_t unpad_add_launch(const PadPlan& p, int64_t b, int64_t m, int64_t n, const float* C_pad,
                              float* C, bool overwrite, cudaStream_t stream, uint64_t* launches) {
   const int64_t total = b * m * n;
-  unpad_add_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(C_pad, C, b * m, n, p.n8,
-                                                                        overwrite ? 1 : 0);
-  const cudaError_t e = cudaGetLastError();
+  const cudaError_t e = launch_chained(unpad_add_kernel, (unsigned)((total + 255) / 256), stream, C_pad, C,
+                                       b * m, n, p.n8, overwrite ? 1 : 0);
   if (e != cudaSuccess) return e;
   ++*launches;
   return cudaSuccess;
