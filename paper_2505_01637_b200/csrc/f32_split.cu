@@ -60,6 +60,47 @@ split_b_kernel(const float* __restrict__ B, uint16_t* __restrict__ B6, int64_t b
   dst[0] = h1; dst[kn] = h3; dst[2 * kn] = h2; dst[3 * kn] = h1; dst[4 * kn] = h2; dst[5 * kn] = h1;
 }
 
+// The same splits, eight neighbouring elements per thread: two 16-byte loads, six 16-byte
+// stores (rows of A with k % 8 == 0, rows of B with n % 8 == 0, 16-byte-aligned pointers).
+__device__ __forceinline__ void split8(const float4 lo, const float4 hi, uint4& t1, uint4& t2, uint4& t3) {
+  const float x[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+  uint32_t w1[4], w2[4], w3[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    uint16_t a1, a2, a3, b1, b2, b3;
+    split3(x[2 * e], a1, a2, a3);
+    split3(x[2 * e + 1], b1, b2, b3);
+    w1[e] = (uint32_t)a1 | ((uint32_t)b1 << 16);
+    w2[e] = (uint32_t)a2 | ((uint32_t)b2 << 16);
+    w3[e] = (uint32_t)a3 | ((uint32_t)b3 << 16);
+  }
+  t1 = make_uint4(w1[0], w1[1], w1[2], w1[3]);
+  t2 = make_uint4(w2[0], w2[1], w2[2], w2[3]);
+  t3 = make_uint4(w3[0], w3[1], w3[2], w3[3]);
+}
+
+__global__ void __launch_bounds__(256)
+split_a8_kernel(const float4* __restrict__ A, uint4* __restrict__ A6, int64_t rows, int64_t k8) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // group of 8 elements
+  if (idx >= rows * k8) return;
+  const int64_t r = idx / k8, g = idx - r * k8;
+  uint4 t1, t2, t3;
+  split8(A[2 * idx], A[2 * idx + 1], t1, t2, t3);
+  uint4* row = A6 + r * 6 * k8 + g;
+  row[0] = t3; row[k8] = t1; row[2 * k8] = t2; row[3 * k8] = t2; row[4 * k8] = t1; row[5 * k8] = t1;
+}
+
+__global__ void __launch_bounds__(256)
+split_b8_kernel(const float4* __restrict__ B, uint4* __restrict__ B6, int64_t b, int64_t kn8) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // group of 8 elements
+  if (idx >= b * kn8) return;
+  const int64_t bb = idx / kn8, rest = idx - bb * kn8;
+  uint4 t1, t2, t3;
+  split8(B[2 * idx], B[2 * idx + 1], t1, t2, t3);
+  uint4* dst = B6 + bb * 6 * kn8 + rest;
+  dst[0] = t1; dst[kn8] = t3; dst[2 * kn8] = t2; dst[3 * kn8] = t1; dst[4 * kn8] = t2; dst[5 * kn8] = t1;
+}
+
 }  // namespace
 
 size_t f32_split_bytes(int64_t b, int64_t m, int64_t k, int64_t n) {
@@ -74,11 +115,21 @@ cudaError_t f32_split_launch(int64_t b, int64_t m, int64_t k, int64_t n, const f
   *A6 = static_cast<uint16_t*>(split);
   *B6 = reinterpret_cast<uint16_t*>(static_cast<char*>(split) + round256((size_t)b * m * k * 12));
   const int64_t ea = b * m * k, eb = b * k * n;
-  split_a_kernel<<<(unsigned)((ea + 255) / 256), 256, 0, stream>>>(A, *A6, b * m, k);
+  const bool a_vec = k % 8 == 0 && reinterpret_cast<uintptr_t>(A) % 16 == 0;
+  const bool b_vec = n % 8 == 0 && reinterpret_cast<uintptr_t>(B) % 16 == 0;
+  if (a_vec)
+    split_a8_kernel<<<(unsigned)((ea / 8 + 255) / 256), 256, 0, stream>>>(
+        reinterpret_cast<const float4*>(A), reinterpret_cast<uint4*>(*A6), b * m, k / 8);
+  else
+    split_a_kernel<<<(unsigned)((ea + 255) / 256), 256, 0, stream>>>(A, *A6, b * m, k);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   ++*launches;
-  split_b_kernel<<<(unsigned)((eb + 255) / 256), 256, 0, stream>>>(B, *B6, b, k, n);
+  if (b_vec)
+    split_b8_kernel<<<(unsigned)((eb / 8 + 255) / 256), 256, 0, stream>>>(
+        reinterpret_cast<const float4*>(B), reinterpret_cast<uint4*>(*B6), b, k * n / 8);
+  else
+    split_b_kernel<<<(unsigned)((eb + 255) / 256), 256, 0, stream>>>(B, *B6, b, k, n);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   ++*launches;
