@@ -209,7 +209,8 @@ size_t workspace_for(int sms, int path, int knob, int64_t b, int64_t m, int64_t 
 
 int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
         const void* B, float* C, void* workspace, size_t workspace_bytes, bool own_scratch,
-        void* stream, bool overwrite = false, bool b_col_major = false) {
+        void* stream, bool overwrite = false, bool b_col_major = false,
+        const KSegments* seg = nullptr) {
   bool empty = false;
   int rc = validate(b, m, k, n, A, B, C, &empty);
   if (rc != MORELLO_OK) return rc;
@@ -318,7 +319,7 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     const GemmPlan plan = gemm_plan(sms, b, m, k, n, split_k);
     if (!plan.supported) return MORELLO_ERR_UNSUPPORTED_PATH;
     e = gemm_launch(st->info, plan, b, m, k, n, static_cast<const uint16_t*>(A),
-                    static_cast<const uint16_t*>(B), C, ws, s, &launches, overwrite, b_col_major);
+                    static_cast<const uint16_t*>(B), C, ws, s, &launches, overwrite, b_col_major, seg);
   } else if (which == SKINNY_STREAM) {
     const StreamPlan plan = stream_plan(sms, b, (int)m, k, n, split_k % kKnobSplitMod,
                                         knob_scratch_reduce(split_k));
@@ -449,13 +450,26 @@ int morello_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n, const f
       st->split_bytes = need;
     }
   }
+  // When the bf16 problem goes to the tensor-core kernels directly and k is a whole number of
+  // their 64-element blocks, only the three terms are stored and the kernels visit them in the
+  // six-product order themselves (half the bytes written by the split); otherwise the six
+  // products are laid out in full and any kernel can run the plain problem of 6k.
+  const void* aligned = reinterpret_cast<const void*>(uintptr_t(4096));   // the split buffers are
+  const bool three = k % 64 == 0 && !staged_wins(b, m, k6, n) &&
+                     select_path(st->info.sms, b, m, k6, n, aligned, aligned, C) == MORELLO_PATH_TCGEN05;
   uint16_t *A6 = nullptr, *B6 = nullptr;
   uint64_t launches = 0;
-  const cudaError_t e = f32_split_launch(b, m, k, n, A, B, st->split, &A6, &B6,
+  const cudaError_t e = f32_split_launch(b, m, k, n, A, B, st->split, !three, &A6, &B6,
                                          static_cast<cudaStream_t>(stream), &launches);
   g_launches.fetch_add(launches, std::memory_order_relaxed);
   if (e != cudaSuccess) return cuda_fail(e);
-  return run(MORELLO_PATH_AUTO, 0, b, m, k6, n, A6, B6, C, nullptr, 0, true, stream);
+  if (!three) return run(MORELLO_PATH_AUTO, 0, b, m, k6, n, A6, B6, C, nullptr, 0, true, stream);
+  // Six segments of k / 64 blocks; stored terms 0, 1, 2 = first, second, third bf16 term.
+  // A: 3, 1, 2, 2, 1, 1 and B: 1, 3, 2, 1, 2, 1 (smallest products first), three bits each.
+  const KSegments seg{(int)(k / 64),
+                      2u | (0u << 3) | (1u << 6) | (1u << 9) | (0u << 12) | (0u << 15),
+                      0u | (2u << 3) | (1u << 6) | (0u << 9) | (1u << 12) | (0u << 15), 3 * k};
+  return run(MORELLO_PATH_TCGEN05, 0, b, m, k6, n, A6, B6, C, nullptr, 0, true, stream, false, false, &seg);
 }
 
 int morello_matmul_accum_host(int64_t b, int64_t m, int64_t k, int64_t n, const void* A_host,

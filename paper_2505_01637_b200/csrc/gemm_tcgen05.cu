@@ -84,6 +84,8 @@ struct GemmParams {
                     // partial[slice][b][m][n]; the slice-ordered reduce kernel adds them and C
   int kb_per_slice; // k blocks per slice
   int64_t bsz;      // batches
+  int seg_blocks;   // > 0: k blocks per segment of the k range (see KSegments); 0: k as stored
+  uint32_t seg_a, seg_b;
   uint32_t* status;
   int overwrite;   // 1: C = product (TMA store) instead of C += product (TMA reduce-add)
   int bt;          // 1: B is stored column-major, [b][n][k]: the K-major operand (boxes of 64 k x 64 columns)
@@ -100,6 +102,14 @@ struct Barriers {
 };
 
 // One unit of work of a thread block (or pair): a tile, or the left / right column half of one.
+// First stored k element of k block kb of the call: kb * 64, or, with segments, block kb's
+// place inside the stored term its segment reads.
+__device__ __forceinline__ int k_coord(int kb, int seg_blocks, uint32_t terms) {
+  if (seg_blocks == 0) return kb * kTileK;
+  const int s = kb / seg_blocks;
+  return ((int)((terms >> (3 * s)) & 7u) * seg_blocks + (kb - s * seg_blocks)) * kTileK;
+}
+
 struct Item {
   int mt, nt, bb;
   int n_off;   // first column of the item inside its tile
@@ -219,6 +229,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
           if (!(ok = mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag, p.status, 1))) break;
           uint8_t* sa = stages + (size_t)stage * S::kStageBytes;
           uint8_t* sb = sa + kBytesA;
+          const int ka = k_coord(kb, p.seg_blocks, p.seg_a), kbb = k_coord(kb, p.seg_blocks, p.seg_b);
           if constexpr (kPair) {
             // Both CTAs' loads complete on the leader's barrier.  Only the leader arrives on
             // it (a local arrive, announcing the bytes of both halves): a load of the peer
@@ -227,23 +238,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const uint32_t full = leader_full + (uint32_t)stage * 8u;
             if (rank == 0)
               mbar_arrive_expect_tx(&bars->full[stage], 2 * stage_tx);
-            tma_load_3d_pair(sa, &map_a, full, kb * kTileK, row0, bb);
+            tma_load_3d_pair(sa, &map_a, full, ka, row0, bb);
 #pragma unroll
             for (int j = 0; j < S::kBoxesB; ++j)
               if (j < boxes_b) {
-                if (p.bt) tma_load_3d_pair(sb + j * kBoxBytesB, &map_b, full, kb * kTileK, col0 + j * 64, bb);
-                else tma_load_3d_pair(sb + j * kBoxBytesB, &map_b, full, col0 + j * 64, kb * kTileK, bb);
+                if (p.bt) tma_load_3d_pair(sb + j * kBoxBytesB, &map_b, full, kbb, col0 + j * 64, bb);
+                else tma_load_3d_pair(sb + j * kBoxBytesB, &map_b, full, col0 + j * 64, kbb, bb);
               }
           } else {
             mbar_arrive_expect_tx(&bars->full[stage], stage_tx);
-            tma_load_3d(sa, &map_a, &bars->full[stage], kb * kTileK, row0, bb);
+            tma_load_3d(sa, &map_a, &bars->full[stage], ka, row0, bb);
 #pragma unroll
             for (int j = 0; j < S::kBoxesB; ++j)
               if (j < boxes_b) {
-                if (p.bt) tma_load_3d(sb + j * kBoxBytesB, &map_b, &bars->full[stage], kb * kTileK,
+                if (p.bt) tma_load_3d(sb + j * kBoxBytesB, &map_b, &bars->full[stage], kbb,
                                       col0 + j * 64, bb);
                 else tma_load_3d(sb + j * kBoxBytesB, &map_b, &bars->full[stage], col0 + j * 64,
-                                 kb * kTileK, bb);
+                                 kbb, bb);
               }
           }
           if (++stage == S::kStages) { stage = 0; phase ^= 1; }
@@ -435,6 +446,8 @@ struct SwapParams {
   int split_k;      // k slices per strip (cluster form: the slices of a strip are one cluster;
                     // otherwise every slice writes its own copy of the output, see the kernel)
   int kb_per_slice; // k blocks per slice
+  int seg_blocks;   // > 0: k blocks per segment of the k range (see KSegments); 0: k as stored
+  uint32_t seg_a, seg_b;
   uint32_t* status;
 };
 
@@ -483,12 +496,13 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     tma_prefetch_descriptor(&map_b);
     const int ahead = min(kb_end, kb_begin + kSwapPrefetchBlocks);
     for (int kb = kb_begin; kb < ahead; ++kb) {
+      const int kbb = k_coord(kb, p.seg_blocks, p.seg_b);
       if (p.bt) {
-        tma_prefetch_l2_3d(&map_b, kb * kTileK, col0, bb);
-        tma_prefetch_l2_3d(&map_b, kb * kTileK, col0 + 64, bb);
+        tma_prefetch_l2_3d(&map_b, kbb, col0, bb);
+        tma_prefetch_l2_3d(&map_b, kbb, col0 + 64, bb);
       } else {
-        tma_prefetch_l2_3d(&map_b, col0, kb * kTileK, bb);
-        tma_prefetch_l2_3d(&map_b, col0 + 64, kb * kTileK, bb);
+        tma_prefetch_l2_3d(&map_b, col0, kbb, bb);
+        tma_prefetch_l2_3d(&map_b, col0 + 64, kbb, bb);
       }
     }
   }
@@ -515,14 +529,15 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         uint8_t* sb = stages + (size_t)stage * S::kStageBytes;
         uint8_t* sa = sb + S::kBytesStrip;
         mbar_arrive_expect_tx(&bars->full[stage], S::kStageBytes);
+        const int ka = k_coord(kb, p.seg_blocks, p.seg_a), kbb = k_coord(kb, p.seg_blocks, p.seg_b);
         if (p.bt) {
-          tma_load_3d(sb, &map_b, &bars->full[stage], kb * kTileK, col0, bb);
-          tma_load_3d(sb + kBoxBytesB, &map_b, &bars->full[stage], kb * kTileK, col0 + 64, bb);
+          tma_load_3d(sb, &map_b, &bars->full[stage], kbb, col0, bb);
+          tma_load_3d(sb + kBoxBytesB, &map_b, &bars->full[stage], kbb, col0 + 64, bb);
         } else {
-          tma_load_3d(sb, &map_b, &bars->full[stage], col0, kb * kTileK, bb);
-          tma_load_3d(sb + kBoxBytesB, &map_b, &bars->full[stage], col0 + 64, kb * kTileK, bb);
+          tma_load_3d(sb, &map_b, &bars->full[stage], col0, kbb, bb);
+          tma_load_3d(sb + kBoxBytesB, &map_b, &bars->full[stage], col0 + 64, kbb, bb);
         }
-        tma_load_3d(sa, &map_a, &bars->full[stage], kb * kTileK, 0, bb);
+        tma_load_3d(sa, &map_a, &bars->full[stage], ka, 0, bb);
         if (++stage == S::kStages) { stage = 0; phase ^= 1; }
       }
       // Every load of this block is in flight: the next kernel's blocks may come in.
@@ -906,7 +921,7 @@ template <bool kPair, int kTileN>
 cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, int64_t n,
                         const CUtensorMap& map_a, const CUtensorMap& map_b,
                         const CUtensorMap& map_c, float* C, bool halves, int ws_split,
-                        bool overwrite, bool bt, cudaStream_t stream) {
+                        bool overwrite, bool bt, const KSegments* seg, cudaStream_t stream) {
   using S = Shape<kPair, kTileN>;
   const cudaError_t attr_err = set_smem_attribute<kPair, kTileN>();
   if (attr_err != cudaSuccess) return attr_err;
@@ -926,6 +941,7 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   p.overwrite = overwrite ? 1 : 0;
   p.bt = bt ? 1 : 0;
   p.bsz = b;
+  if (seg) { p.seg_blocks = seg->blocks; p.seg_a = seg->a_terms; p.seg_b = seg->b_terms; }
   p.ws_split = std::max(1, ws_split);
   p.kb_per_slice = (p.k_blocks + p.ws_split - 1) / p.ws_split;
   if (p.ws_split > 1) {      // map_c covers the partial sums; every item stores its own
@@ -974,7 +990,7 @@ namespace {
 template <int kRowsA, bool kClusterK>
 cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_t m, int64_t k, int64_t n,
                              const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
-                             bool overwrite, bool bt, cudaStream_t stream) {
+                             bool overwrite, bool bt, const KSegments* seg, cudaStream_t stream) {
   using S = SwapShape<kRowsA>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
@@ -992,6 +1008,7 @@ cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_
   p.split_k = std::max(1, split);
   p.kb_per_slice = (p.k_blocks + p.split_k - 1) / p.split_k;
   p.status = dev.status;
+  if (seg) { p.seg_blocks = seg->blocks; p.seg_a = seg->a_terms; p.seg_b = seg->b_terms; }
   const int64_t strips = (n + kSwapStripCols - 1) / kSwapStripCols;
   // grid.y carries the batch index (the planner keeps batches beyond a grid dimension off
   // this kernel).
@@ -1023,18 +1040,19 @@ cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_
 template <int kRowsA>
 cudaError_t launch_swap(const DeviceInfo& dev, int split, int ws_split, int64_t b, int64_t m, int64_t k,
                         int64_t n, const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
-                        bool overwrite, bool bt, cudaStream_t stream) {
+                        bool overwrite, bool bt, const KSegments* seg, cudaStream_t stream) {
   return split > 1 ? launch_swap_form<kRowsA, true>(dev, split, b, m, k, n, map_a, map_b, C, overwrite,
-                                                    bt, stream)
+                                                    bt, seg, stream)
                    : launch_swap_form<kRowsA, false>(dev, ws_split, b, m, k, n, map_a, map_b, C,
-                                                     overwrite, bt, stream);
+                                                     overwrite, bt, seg, stream);
 }
 
 }  // namespace
 
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m, int64_t k,
                         int64_t n, const uint16_t* A, const uint16_t* B, float* C, float* workspace,
-                        cudaStream_t stream, uint64_t* launches, bool overwrite, bool bt) {
+                        cudaStream_t stream, uint64_t* launches, bool overwrite, bool bt,
+                        const KSegments* seg) {
   // With k slices through the workspace the kernels write partial[slice][b][m][n] there (plain
   // stores) and the reduce launch below adds the slices and C.
   const bool sliced = plan.ws_split > 1;
@@ -1042,21 +1060,24 @@ cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, 
   float* out = sliced ? workspace : C;
   const bool out_overwrite = sliced ? true : overwrite;
   CUtensorMap map_a, map_b, map_c;
-  cudaError_t e = get_maps(MapKey{A, B, out, b, m, k, n, bt, sliced ? plan.ws_split * b : b}, &map_a,
-                           &map_b, &map_c);
+  // With segments the stored operands are shorter along k than the call's k range.
+  if (seg && (seg->blocks <= 0 || k % (64ll * seg->blocks) != 0 || k / (64ll * seg->blocks) > 8))
+    return cudaErrorInvalidValue;
+  cudaError_t e = get_maps(MapKey{A, B, out, b, m, seg ? seg->k_stored : k, n, bt, sliced ? plan.ws_split * b : b},
+                           &map_a, &map_b, &map_c);
   if (e != cudaSuccess) return e;
   const int code = plan.form * 1000 + plan.tile_n;
   const int wss = plan.ws_split;
   switch (code) {
-    case 3016: e = launch_swap<16>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, stream); break;
-    case 3032: e = launch_swap<32>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, stream); break;
-    case 3048: e = launch_swap<48>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, stream); break;
-    case 3064: e = launch_swap<64>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, stream); break;
-    case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, stream); break;
-    case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, stream); break;
-    case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, stream); break;
-    case 2128: e = launch_gemm<true, 128>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, stream); break;
-    case 2256: e = launch_gemm<true, 256>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, stream); break;
+    case 3016: e = launch_swap<16>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, seg, stream); break;
+    case 3032: e = launch_swap<32>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, seg, stream); break;
+    case 3048: e = launch_swap<48>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, seg, stream); break;
+    case 3064: e = launch_swap<64>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, seg, stream); break;
+    case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, seg, stream); break;
+    case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, seg, stream); break;
+    case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, seg, stream); break;
+    case 2128: e = launch_gemm<true, 128>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, seg, stream); break;
+    case 2256: e = launch_gemm<true, 256>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, seg, stream); break;
     default: return cudaErrorInvalidValue;
   }
   if (e != cudaSuccess) return e;

@@ -80,7 +80,7 @@ cudaError_t stream_launch(const DeviceInfo& dev, const StreamPlan& plan, int64_t
 size_t f32_split_bytes(int64_t b, int64_t m, int64_t k, int64_t n);
 // Enqueues the two split kernels; *A6 and *B6 point into `split` afterwards.
 cudaError_t f32_split_launch(int64_t b, int64_t m, int64_t k, int64_t n, const float* A, const float* B,
-                             void* split, uint16_t** A6, uint16_t** B6, cudaStream_t stream,
+                             void* split, bool six, uint16_t** A6, uint16_t** B6, cudaStream_t stream,
                              uint64_t* launches);
 
 // ---- zero-padded copies of operands the TMA engine cannot address --------------
@@ -117,12 +117,21 @@ bool gemm_shape_supported(int64_t b, int64_t m, int64_t k, int64_t n, const void
 // tiles whole], the first two parts 0 = by shape; with form 3 the second part is the number of k
 // slices (0 = by shape, 1, 2, 4 or 8).
 GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob);
+// The k range as a sequence of up to 8 equal segments, each reading one of the stored k ranges
+// of A and of B (float32 inputs: six products of three stored terms each, see f32_split.cu):
+// segment s covers k blocks [s * blocks, (s + 1) * blocks) of the call and reads stored blocks
+// term * blocks + ..., term = 3 bits of a_terms / b_terms at position 3 s.
+struct KSegments {
+  int blocks;            // 64-element k blocks per segment
+  uint32_t a_terms, b_terms;
+  int64_t k_stored;      // k extent of the stored A and B (terms x blocks x 64)
+};
 // CTA pairs (cta_group::2) the current device can hold at once.
 int gemm_pair_units(int sms);
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m,
                         int64_t k, int64_t n, const uint16_t* A, const uint16_t* B, float* C,
                         float* workspace, cudaStream_t stream, uint64_t* launches,
-                        bool overwrite = false, bool b_col_major = false);
+                        bool overwrite = false, bool b_col_major = false, const KSegments* seg = nullptr);
 
 // ---- B stored column-major where the TMA engine cannot address it ------------
 // C[b, i, j] (+)= sum_p A[b, i, p] * Bt[b, j, p]: one warp per output column, lanes stride over

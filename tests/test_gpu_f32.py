@@ -8,6 +8,7 @@ import torch
 
 import oracle
 from paper_2505_01637_b200 import binding as mb
+from paper_2505_01637_b200 import workloads as w
 
 from gpu_util import assert_bit_exact, assert_within_tolerance
 
@@ -95,3 +96,33 @@ def test_f32_empty_and_bad_arguments():
     with pytest.raises(mb.MorelloError) as e:
         mb.morello_matmul_accum_f32(1, -2, 4, 8, dA, dA, dC)
     assert e.value.status == mb.MORELLO_ERR_INVALID_SHAPE
+
+
+@pytest.mark.parametrize("shape", [
+    (1, 256, 512, 512),      # tile kernel
+    (2, 16, 1024, 1024),     # operand-swapped kernel
+    (1, 8, 4096, 256),       # ... with k slices inside a cluster
+    (1, 300, 4096, 264),     # tile kernel with k slices through the workspace
+    (1, 64, 64, 128),        # one k block per term
+])
+def test_f32_three_stored_terms_equal_the_six_term_problem(shape):
+    """With k % 64 == 0 the library stores the three bf16 terms of A and B once and lets the
+    tensor kernels visit them in the six-product order.  The same six products laid out in
+    full on the host and run as a plain bf16 problem of 6k must give the same bits."""
+    b, m, k, n = shape
+    A, B, C = _draw(shape, 21 + sum(shape), "wide")
+
+    def terms(x):
+        h1 = w.f32_to_bf16_rne(x)
+        r1 = x - w.bf16_to_f32(h1)
+        h2 = w.f32_to_bf16_rne(r1)
+        r2 = r1 - w.bf16_to_f32(h2)
+        return h1, h2, w.f32_to_bf16_rne(r2)
+
+    a1, a2, a3 = terms(A)
+    b1, b2, b3 = terms(B)
+    A6 = np.ascontiguousarray(np.concatenate([a3, a1, a2, a2, a1, a1], axis=2))
+    B6 = np.ascontiguousarray(np.concatenate([b1, b3, b2, b1, b2, b1], axis=1))
+    from gpu_util import gpu_run
+    plain = gpu_run(A6, B6, C)
+    assert np.array_equal(_gpu(shape, A, B, C).view(np.uint32), plain.view(np.uint32))
