@@ -52,6 +52,8 @@ def _load():
         lib.oracle_matmul_accum_f32.restype = ctypes.c_int
         lib.oracle_matmul_accum_bt.argtypes = [i64, i64, i64, i64, vp, vp, vp]
         lib.oracle_matmul_accum_bt.restype = None
+        lib.oracle_matmul_accum_packed_b.argtypes = [i64, i64, i64, i64, i64, vp, vp, vp]
+        lib.oracle_matmul_accum_packed_b.restype = None
         lib.oracle_num_threads.restype = ctypes.c_int
         lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
         _lib = lib
@@ -125,6 +127,18 @@ def matmul_accum_bt(b, m, k, n, A, Bt, C) -> np.ndarray:
     out = np.array(C, dtype=np.float32, copy=True, order="C")
     assert out.size == b * m * n
     _load().oracle_matmul_accum_bt(b, m, k, n, _ptr(A), _ptr(Bt), _ptr(out))
+    return out
+
+
+def matmul_accum_packed_b(strip, b, m, k, n, A, Bp, C) -> np.ndarray:
+    """B given packed in strips of `strip` columns (Bp[b][ceil(n/strip)][k][strip], bf16 bit
+    patterns, last strip padded): returns C + A x B."""
+    strips = (n + strip - 1) // strip
+    assert Bp.dtype == np.uint16 and Bp.flags.c_contiguous and Bp.size == b * strips * k * strip
+    assert A.dtype == np.uint16 and A.flags.c_contiguous and A.size == b * m * k
+    out = np.array(C, dtype=np.float32, copy=True, order="C")
+    assert out.size == b * m * n
+    _load().oracle_matmul_accum_packed_b(strip, b, m, k, n, _ptr(A), _ptr(Bp), _ptr(out))
     return out
 
 

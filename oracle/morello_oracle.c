@@ -260,3 +260,35 @@ void oracle_matmul_accum_bt(int64_t b, int64_t m, int64_t k, int64_t n,
         }
     }
 }
+
+/*
+ * The bf16 operation with the right-hand side in a packed layout (paper Section 2.4.2: a
+ * layout may carry a strip dimension of size s on one logical dimension; Goto-style packing).
+ * Here the strips run over the column index j: strip j / s holds columns [s (j / s), s (j / s) + s)
+ * of every row, row-major inside the strip, and the strips follow one another,
+ *
+ *     offset(p, j) = (j / s) * k * s  +  p * s  +  (j mod s),      Bp[b][ceil(n / s)][k][s]
+ *
+ * (the last strip is padded to s columns; the padding is never read).
+ *
+ *     C[b,i,j]  <-  C[b,i,j] + sum_{p=0}^{k-1} A[b,i,p] * Bp[b][j / s][p][j mod s]
+ *
+ * Same arithmetic as everywhere above (double accumulation of exact products in increasing p,
+ * one rounding); only the indexing of the right-hand side differs.
+ */
+void oracle_matmul_accum_packed_b(int64_t s, int64_t b, int64_t m, int64_t k, int64_t n,
+                                  const uint16_t *A, const uint16_t *Bp, float *C)
+{
+    const int64_t strips = (n + s - 1) / s;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < b * m; ++r) {
+        const int64_t bb = r / m;
+        for (int64_t j = 0; j < n; ++j) {
+            double sum = (double)C[r * n + j];
+            const uint16_t *col = Bp + ((bb * strips + j / s) * k) * s + (j % s);
+            for (int64_t p = 0; p < k; ++p)
+                sum += bf16_to_double(A[r * k + p]) * bf16_to_double(col[p * s]);
+            C[r * n + j] = (float)sum;
+        }
+    }
+}

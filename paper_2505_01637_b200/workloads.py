@@ -155,3 +155,13 @@ def sample_rows(b, m, seed, edge=128, stride=64):
         for i0 in range(0, m, stride):
             rows.add(beta * m + i0 + int(rng.integers(0, min(stride, m - i0))))
     return np.array(sorted(rows), dtype=np.int64)
+
+
+def pack_b(B: np.ndarray, strip: int, fill: int = 0) -> np.ndarray:
+    """B[b][k][n] (any 16-bit patterns) -> the packed layout Bp[b][ceil(n/strip)][k][strip]:
+    strips of `strip` columns, row-major inside a strip, the last strip padded with `fill`."""
+    b, k, n = B.shape
+    strips = (n + strip - 1) // strip
+    padded = np.full((b, k, strips * strip), fill, dtype=B.dtype)
+    padded[:, :, :n] = B
+    return np.ascontiguousarray(padded.reshape(b, k, strips, strip).transpose(0, 2, 1, 3))

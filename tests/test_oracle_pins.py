@@ -410,3 +410,33 @@ def test_colmajor_oracle_one_hot_pins_the_indexing():
     want[1, :, 2] += -3.0 * Av[1, :, 3]
     got = oracle.matmul_accum_bt(b, m, k, n, as_bf16(Av), as_bf16(Bt1), C)
     assert np.array_equal(got, want)
+
+
+# ------------------------------------------------ packed right-hand side (Section 2.4.2: a strip
+# dimension of size s on the column index): pinned to the offset formula written out, to a
+# hand-computed offset, and to the row-major oracle
+def test_packed_oracle_follows_the_offset_formula():
+    for (s, b, m, k, n) in [(4, 2, 3, 5, 10), (8, 1, 2, 7, 8), (64, 1, 2, 3, 70), (16, 3, 1, 9, 5)]:
+        A, B, C = w.make(b, m, k, n, seed=31 + s, ab="uniform", c="normal")
+        strips = (n + s - 1) // s
+        Bp = np.full(b * strips * k * s, 0x7FC0, np.uint16)          # padding = NaN patterns: never read
+        for bb in range(b):
+            for p in range(k):
+                for j in range(n):
+                    Bp[bb * strips * k * s + (j // s) * k * s + p * s + (j % s)] = B[bb, p, j]
+        got = oracle.matmul_accum_packed_b(s, b, m, k, n, A, Bp, C)
+        assert np.array_equal(bits(got), bits(oracle.matmul_accum(b, m, k, n, A, B, C)))
+        assert np.array_equal(w.pack_b(B, s, fill=0x7FC0).reshape(-1), Bp)   # the test helper packs the same way
+
+
+def test_packed_oracle_one_hot_at_a_hand_computed_offset():
+    s, b, m, k, n = 4, 1, 3, 5, 10                       # 3 strips of 4 columns, 5 rows each
+    rng = np.random.default_rng(11)
+    Av = rng.integers(-100, 101, size=(b, m, k)).astype(np.float32)
+    C = rng.integers(-50, 51, size=(b, m, n)).astype(np.float32)
+    Bp = np.zeros(3 * 5 * 4, np.float32)
+    Bp[1 * 20 + 3 * 4 + 2] = -3.0                        # strip 1, row p = 3, column 2 of the strip: j = 6
+    want = C.copy()
+    want[0, :, 6] += -3.0 * Av[0, :, 3]
+    got = oracle.matmul_accum_packed_b(s, b, m, k, n, as_bf16(Av), as_bf16(Bp), C)
+    assert np.array_equal(got, want)
