@@ -125,6 +125,26 @@ int morello_matmul_accum_colmajor_b(int tile, int64_t b, int64_t m, int64_t k, i
                                     const void* A, const void* Bt, float* C, void* stream);
 
 /*
+ * MatmulAccum with B in a packed layout (Section 2.4.2 of the paper: a layout may carry a strip
+ * dimension of size s on a logical dimension -- Goto-style packing): the columns of B are cut
+ * into strips of `strip`, each strip stored row-major and the strips one after another,
+ *
+ *     Bp[b][ceil(n / strip)][k][strip] bf16,    B[b,p,j] = Bp[b][j / strip][p][j mod strip]
+ *
+ * (the last strip is padded to `strip` columns; the padding is never used, whatever it holds).
+ *
+ *     C[b,i,j]  <-  C[b,i,j] + sum_{p<k} A[b,i,p] * B[b,p,j]
+ *
+ * A and C as everywhere else.  With strip % 64 == 0, k % 8 == 0, n % 8 == 0 and 16-byte-aligned
+ * pointers the tensor-core kernels run it (a 64-column box of a strip is one contiguous 8 KiB
+ * read); anything else runs on a plain one-thread-per-output kernel.  strip == 1 is the
+ * column-major layout.  Scratch as in morello_matmul_accum.  Same status codes, asynchronous on
+ * `stream`, deterministic.
+ */
+int morello_matmul_accum_packed_b(int strip, int64_t b, int64_t m, int64_t k, int64_t n,
+                                  const void* A, const void* Bp, float* C, void* stream);
+
+/*
  * MatmulAccum on float32 inputs (the paper's other benchmark, Section 7, is a float32
  * 2048-square matrix multiplication): A[b][m][k], B[b][k][n] and C[b][m][n] all f32, dense
  * row-major device pointers, 4-byte aligned; C += A x B.

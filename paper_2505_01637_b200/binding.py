@@ -39,6 +39,7 @@ SIGNATURES = {
                                      _vp, _sz, _vp]),
     "morello_matmul_accum_f32": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
     "morello_matmul_accum_colmajor_b": (_int, [_int, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
+    "morello_matmul_accum_packed_b": (_int, [_int, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
     "morello_workspace_bytes": (_sz, [_i64, _i64, _i64, _i64]),
     "morello_matmul_accum_ws": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _sz, _vp]),
     "morello_matmul_accum_host": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp]),
@@ -143,6 +144,13 @@ def morello_matmul_accum_colmajor_b(tile, b, m, k, n, A, Bt, C, stream=None) -> 
     _check(lib().morello_matmul_accum_colmajor_b(tile, b, m, k, n, _addr(A), _addr(Bt), _addr(C),
                                                  _stream(stream)),
            "morello_matmul_accum_colmajor_b")
+
+
+def morello_matmul_accum_packed_b(strip, b, m, k, n, A, Bp, C, stream=None) -> None:
+    """C += A x B with B packed in strips of `strip` columns: Bp[b][ceil(n/strip)][k][strip]."""
+    _check(lib().morello_matmul_accum_packed_b(strip, b, m, k, n, _addr(A), _addr(Bp), _addr(C),
+                                               _stream(stream)),
+           "morello_matmul_accum_packed_b")
 
 
 def morello_workspace_bytes(b, m, k, n) -> int:

@@ -209,7 +209,7 @@ size_t workspace_for(int sms, int path, int knob, int64_t b, int64_t m, int64_t 
 
 int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
         const void* B, float* C, void* workspace, size_t workspace_bytes, bool own_scratch,
-        void* stream, bool overwrite = false, bool b_col_major = false,
+        void* stream, bool overwrite = false, int b_layout = 0,
         const KSegments* seg = nullptr) {
   bool empty = false;
   int rc = validate(b, m, k, n, A, B, C, &empty);
@@ -234,13 +234,17 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     return MORELLO_OK;
   }
 
+  // b_layout: 0 row-major B, 1 column-major, otherwise the strip size of a packed B.
+  const bool b_col_major = b_layout != 0;     // any layout but row-major: tensor kernels or a fallback
   bool bt_fallback = false;
   bool staged = false;   // through zero-padded copies of the operands (see pad.cu)
   if (b_col_major) {
-    // B as [b][n][k]: the tensor-core kernels when the TMA engine can address the operands,
-    // else the one-warp-per-column kernel.  The FMA streaming kernels read B by rows only.
+    // B as [b][n][k] or packed in strips: the tensor-core kernels when the TMA engine can
+    // address the operands (a packed B needs strips that are multiples of their 64-column
+    // boxes), else a plain kernel.  The FMA streaming kernels read B by rows only.
     if (path == MORELLO_PATH_SKINNY) return MORELLO_ERR_UNSUPPORTED_PATH;
-    const bool tc = gemm_shape_supported(b, m, k, n, A, B, C);
+    const bool tc = gemm_shape_supported(b, m, k, n, A, B, C) && (b_layout == 1 || b_layout % 64 == 0) &&
+                    (b_layout == 1 || b * ((n + b_layout - 1) / b_layout) < (1ll << 31));
     if (path == MORELLO_PATH_TCGEN05 && !tc) return MORELLO_ERR_UNSUPPORTED_PATH;
     path = MORELLO_PATH_TCGEN05;
     bt_fallback = !tc;
@@ -312,6 +316,9 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
                       &launches, pad.stage_c ? true : overwrite);
     if (e == cudaSuccess && pad.stage_c)
       e = unpad_add_launch(pad, b, m, n, c_pad, C, overwrite, s, &launches);
+  } else if (bt_fallback && b_layout != 1) {
+    e = packed_fallback_launch(b_layout, b, m, k, n, static_cast<const uint16_t*>(A),
+                               static_cast<const uint16_t*>(B), C, overwrite, s, &launches);
   } else if (bt_fallback) {
     e = colmajor_fallback_launch(b, m, k, n, static_cast<const uint16_t*>(A),
                                  static_cast<const uint16_t*>(B), C, overwrite, s, &launches);
@@ -319,7 +326,7 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     const GemmPlan plan = gemm_plan(sms, b, m, k, n, split_k);
     if (!plan.supported) return MORELLO_ERR_UNSUPPORTED_PATH;
     e = gemm_launch(st->info, plan, b, m, k, n, static_cast<const uint16_t*>(A),
-                    static_cast<const uint16_t*>(B), C, ws, s, &launches, overwrite, b_col_major, seg);
+                    static_cast<const uint16_t*>(B), C, ws, s, &launches, overwrite, b_layout, seg);
   } else if (which == SKINNY_STREAM) {
     const StreamPlan plan = stream_plan(sms, b, (int)m, k, n, split_k % kKnobSplitMod,
                                         knob_scratch_reduce(split_k));
@@ -413,6 +420,17 @@ int morello_matmul_accum_colmajor_b(int tile, int64_t b, int64_t m, int64_t k, i
   return run(MORELLO_PATH_AUTO, tile, b, m, k, n, A, Bt, C, nullptr, 0, true, stream, false, true);
 }
 
+int morello_matmul_accum_packed_b(int strip, int64_t b, int64_t m, int64_t k, int64_t n,
+                                  const void* A, const void* Bp, float* C, void* stream) {
+  if (strip < 1) return MORELLO_ERR_INVALID_SHAPE;
+  int64_t t;
+  if (n > 0 && (mul_overflows((n + strip - 1) / strip, strip, &t) || mul_overflows(t, k > 0 ? k : 1, &t) ||
+                mul_overflows(t, b > 0 ? b : 1, &t) || mul_overflows(t, 2, &t)))
+    return MORELLO_ERR_INVALID_SHAPE;
+  // A strip of one column is the column-major layout; the code 1 means exactly that below.
+  return run(MORELLO_PATH_AUTO, 0, b, m, k, n, A, Bp, C, nullptr, 0, true, stream, false, strip);
+}
+
 int morello_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n, const float* A,
                              const float* B, float* C, void* stream) {
   if (b < 0 || m < 0 || k < 0 || n < 0) return MORELLO_ERR_INVALID_SHAPE;
@@ -469,7 +487,7 @@ int morello_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n, const f
   const KSegments seg{(int)(k / 64),
                       2u | (0u << 3) | (1u << 6) | (1u << 9) | (0u << 12) | (0u << 15),
                       0u | (2u << 3) | (1u << 6) | (0u << 9) | (1u << 12) | (0u << 15), 3 * k};
-  return run(MORELLO_PATH_TCGEN05, 0, b, m, k6, n, A6, B6, C, nullptr, 0, true, stream, false, false, &seg);
+  return run(MORELLO_PATH_TCGEN05, 0, b, m, k6, n, A6, B6, C, nullptr, 0, true, stream, false, 0, &seg);
 }
 
 int morello_matmul_accum_host(int64_t b, int64_t m, int64_t k, int64_t n, const void* A_host,

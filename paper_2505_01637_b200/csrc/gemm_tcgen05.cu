@@ -86,6 +86,8 @@ struct GemmParams {
   int64_t bsz;      // batches
   int seg_blocks;   // > 0: k blocks per segment of the k range (see KSegments); 0: k as stored
   uint32_t seg_a, seg_b;
+  int pack_strip;   // > 0: B is packed in strips of this many columns (a multiple of 64)
+  int pack_strips;  // strips per batch
   uint32_t* status;
   int overwrite;   // 1: C = product (TMA store) instead of C += product (TMA reduce-add)
   int bt;          // 1: B is stored column-major, [b][n][k]: the K-major operand (boxes of 64 k x 64 columns)
@@ -108,6 +110,25 @@ __device__ __forceinline__ int k_coord(int kb, int seg_blocks, uint32_t terms) {
   if (seg_blocks == 0) return kb * kTileK;
   const int s = kb / seg_blocks;
   return ((int)((terms >> (3 * s)) & 7u) * seg_blocks + (kb - s * seg_blocks)) * kTileK;
+}
+
+// TMA coordinates of the 64-column box of B at (first column `col`, first k element `kc`) of
+// batch bb: row-major B is {n, k, b}; column-major {k, n, b}; packed in strips of `strip`
+// columns {strip, k, b * strips} (the strip index folded into the batch coordinate).
+struct BBox { int x, y, z; };
+__device__ __forceinline__ BBox b_box(int bt, int strip, int strips, int col, int kc, int bb) {
+  if (bt) return BBox{kc, col, bb};
+  if (strip) {
+    const int st = col / strip;
+    return BBox{col - st * strip, kc, bb * strips + st};
+  }
+  return BBox{col, kc, bb};
+}
+// The same box at another k: only the k coordinate changes (the strip arithmetic, a division,
+// is done once per item, outside the k loop).
+__device__ __forceinline__ BBox at_k(BBox box, int bt, int kc) {
+  if (bt) box.x = kc; else box.y = kc;
+  return box;
 }
 
 struct Item {
@@ -225,6 +246,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int boxes_b = cols_b / 64;
         const int col0 = it.nt * kTileN + it.n_off + (int)rank * cols_b;
         const uint32_t stage_tx = (uint32_t)(boxes_b * kBoxBytesB + p.a_box_rows * (kTileK * 2));
+        BBox boxes[S::kBoxesB];
+#pragma unroll
+        for (int j = 0; j < S::kBoxesB; ++j)
+          boxes[j] = b_box(p.bt, p.pack_strip, p.pack_strips, col0 + j * 64, 0, bb);
         for (int kb = it.kb0; kb < it.kb1; ++kb) {
           if (!(ok = mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag, p.status, 1))) break;
           uint8_t* sa = stages + (size_t)stage * S::kStageBytes;
@@ -242,8 +267,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
             for (int j = 0; j < S::kBoxesB; ++j)
               if (j < boxes_b) {
-                if (p.bt) tma_load_3d_pair(sb + j * kBoxBytesB, &map_b, full, kbb, col0 + j * 64, bb);
-                else tma_load_3d_pair(sb + j * kBoxBytesB, &map_b, full, col0 + j * 64, kbb, bb);
+                const BBox c = at_k(boxes[j], p.bt, kbb);
+                tma_load_3d_pair(sb + j * kBoxBytesB, &map_b, full, c.x, c.y, c.z);
               }
           } else {
             mbar_arrive_expect_tx(&bars->full[stage], stage_tx);
@@ -251,10 +276,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
             for (int j = 0; j < S::kBoxesB; ++j)
               if (j < boxes_b) {
-                if (p.bt) tma_load_3d(sb + j * kBoxBytesB, &map_b, &bars->full[stage], kbb,
-                                      col0 + j * 64, bb);
-                else tma_load_3d(sb + j * kBoxBytesB, &map_b, &bars->full[stage], col0 + j * 64,
-                                 kbb, bb);
+                const BBox c = at_k(boxes[j], p.bt, kbb);
+                tma_load_3d(sb + j * kBoxBytesB, &map_b, &bars->full[stage], c.x, c.y, c.z);
               }
           }
           if (++stage == S::kStages) { stage = 0; phase ^= 1; }
@@ -448,6 +471,8 @@ struct SwapParams {
   int kb_per_slice; // k blocks per slice
   int seg_blocks;   // > 0: k blocks per segment of the k range (see KSegments); 0: k as stored
   uint32_t seg_a, seg_b;
+  int pack_strip;   // > 0: B is packed in strips of this many columns (a multiple of 64)
+  int pack_strips;  // strips per batch
   uint32_t* status;
 };
 
@@ -495,15 +520,13 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     tma_prefetch_descriptor(&map_a);
     tma_prefetch_descriptor(&map_b);
     const int ahead = min(kb_end, kb_begin + kSwapPrefetchBlocks);
+    const BBox box0 = b_box(p.bt, p.pack_strip, p.pack_strips, col0, 0, bb);
+    const BBox box1 = b_box(p.bt, p.pack_strip, p.pack_strips, col0 + 64, 0, bb);
     for (int kb = kb_begin; kb < ahead; ++kb) {
       const int kbb = k_coord(kb, p.seg_blocks, p.seg_b);
-      if (p.bt) {
-        tma_prefetch_l2_3d(&map_b, kbb, col0, bb);
-        tma_prefetch_l2_3d(&map_b, kbb, col0 + 64, bb);
-      } else {
-        tma_prefetch_l2_3d(&map_b, col0, kbb, bb);
-        tma_prefetch_l2_3d(&map_b, col0 + 64, kbb, bb);
-      }
+      const BBox c0 = at_k(box0, p.bt, kbb), c1 = at_k(box1, p.bt, kbb);
+      tma_prefetch_l2_3d(&map_b, c0.x, c0.y, c0.z);
+      tma_prefetch_l2_3d(&map_b, c1.x, c1.y, c1.z);
     }
   }
   if (warp == 1) {
@@ -524,19 +547,17 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     if (elect_one()) {
       int stage = 0;
       uint32_t phase = 0;
+      const BBox box0 = b_box(p.bt, p.pack_strip, p.pack_strips, col0, 0, bb);
+      const BBox box1 = b_box(p.bt, p.pack_strip, p.pack_strips, col0 + 64, 0, bb);
       for (int kb = kb_begin; kb < kb_end; ++kb) {
         if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag, p.status, 8)) break;
         uint8_t* sb = stages + (size_t)stage * S::kStageBytes;
         uint8_t* sa = sb + S::kBytesStrip;
         mbar_arrive_expect_tx(&bars->full[stage], S::kStageBytes);
         const int ka = k_coord(kb, p.seg_blocks, p.seg_a), kbb = k_coord(kb, p.seg_blocks, p.seg_b);
-        if (p.bt) {
-          tma_load_3d(sb, &map_b, &bars->full[stage], kbb, col0, bb);
-          tma_load_3d(sb + kBoxBytesB, &map_b, &bars->full[stage], kbb, col0 + 64, bb);
-        } else {
-          tma_load_3d(sb, &map_b, &bars->full[stage], col0, kbb, bb);
-          tma_load_3d(sb + kBoxBytesB, &map_b, &bars->full[stage], col0 + 64, kbb, bb);
-        }
+        const BBox c0 = at_k(box0, p.bt, kbb), c1 = at_k(box1, p.bt, kbb);
+        tma_load_3d(sb, &map_b, &bars->full[stage], c0.x, c0.y, c0.z);
+        tma_load_3d(sb + kBoxBytesB, &map_b, &bars->full[stage], c1.x, c1.y, c1.z);
         tma_load_3d(sa, &map_a, &bars->full[stage], ka, 0, bb);
         if (++stage == S::kStages) { stage = 0; phase ^= 1; }
       }
@@ -657,7 +678,7 @@ struct MapKey {
   const void* b;
   const void* c;
   int64_t bsz, m, k, n;
-  bool bt;   // B column-major
+  int bt;    // layout of B: 0 row-major, 1 column-major, >= 64 packed in strips of that many columns
   int64_t c_bsz;   // batches of the output map: bsz, or slices x bsz when c is the workspace
   bool operator==(const MapKey& o) const {
     return a == o.a && b == o.b && c == o.c && bsz == o.bsz && m == o.m && k == o.k && n == o.n &&
@@ -698,10 +719,14 @@ cudaError_t get_maps(const MapKey& key, CUtensorMap* ma, CUtensorMap* mb, CUtens
   if (err != cudaSuccess) return err;
   // Either way a box is 64 x 64 elements with 128-byte rows: [k][n] gives 64 k rows of 64
   // columns, [n][k] gives 64 columns (rows of the stored matrix) of 64 k.
-  if (key.bt)
+  if (key.bt == 1)
     err = make_tensor_map_3d(&e.map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, key.b, (uint64_t)key.k,
                              (uint64_t)key.n, (uint64_t)key.bsz, kTileK, 64,
                              CU_TENSOR_MAP_SWIZZLE_128B);
+  else if (key.bt >= 64)   // packed: {strip, k, b x strips}; a box is again 64 k rows of 64 columns
+    err = make_tensor_map_3d(&e.map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, key.b, (uint64_t)key.bt,
+                             (uint64_t)key.k, (uint64_t)(key.bsz * ((key.n + key.bt - 1) / key.bt)), 64,
+                             kTileK, CU_TENSOR_MAP_SWIZZLE_128B);
   else
     err = make_tensor_map_3d(&e.map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, key.b, (uint64_t)key.n,
                              (uint64_t)key.k, (uint64_t)key.bsz, 64, kTileK,
@@ -921,7 +946,7 @@ template <bool kPair, int kTileN>
 cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, int64_t n,
                         const CUtensorMap& map_a, const CUtensorMap& map_b,
                         const CUtensorMap& map_c, float* C, bool halves, int ws_split,
-                        bool overwrite, bool bt, const KSegments* seg, cudaStream_t stream) {
+                        bool overwrite, int bt, const KSegments* seg, cudaStream_t stream) {
   using S = Shape<kPair, kTileN>;
   const cudaError_t attr_err = set_smem_attribute<kPair, kTileN>();
   if (attr_err != cudaSuccess) return attr_err;
@@ -939,7 +964,9 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   p.status = dev.status;
   p.a_box_rows = a_box_rows(m);
   p.overwrite = overwrite ? 1 : 0;
-  p.bt = bt ? 1 : 0;
+  p.bt = bt == 1 ? 1 : 0;
+  p.pack_strip = bt >= 64 ? bt : 0;
+  p.pack_strips = bt >= 64 ? (int)((n + bt - 1) / bt) : 0;
   p.bsz = b;
   if (seg) { p.seg_blocks = seg->blocks; p.seg_a = seg->a_terms; p.seg_b = seg->b_terms; }
   p.ws_split = std::max(1, ws_split);
@@ -990,7 +1017,7 @@ namespace {
 template <int kRowsA, bool kClusterK>
 cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_t m, int64_t k, int64_t n,
                              const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
-                             bool overwrite, bool bt, const KSegments* seg, cudaStream_t stream) {
+                             bool overwrite, int bt, const KSegments* seg, cudaStream_t stream) {
   using S = SwapShape<kRowsA>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
@@ -1000,7 +1027,9 @@ cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_
   });
   if (attr_err != cudaSuccess) return attr_err;
   SwapParams p{};
-  p.bt = bt ? 1 : 0;
+  p.bt = bt == 1 ? 1 : 0;
+  p.pack_strip = bt >= 64 ? bt : 0;
+  p.pack_strips = bt >= 64 ? (int)((n + bt - 1) / bt) : 0;
   p.overwrite = overwrite ? 1 : 0;
   p.m = m; p.n = n;
   p.c_batch = m * n;
@@ -1040,7 +1069,7 @@ cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_
 template <int kRowsA>
 cudaError_t launch_swap(const DeviceInfo& dev, int split, int ws_split, int64_t b, int64_t m, int64_t k,
                         int64_t n, const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
-                        bool overwrite, bool bt, const KSegments* seg, cudaStream_t stream) {
+                        bool overwrite, int bt, const KSegments* seg, cudaStream_t stream) {
   return split > 1 ? launch_swap_form<kRowsA, true>(dev, split, b, m, k, n, map_a, map_b, C, overwrite,
                                                     bt, seg, stream)
                    : launch_swap_form<kRowsA, false>(dev, ws_split, b, m, k, n, map_a, map_b, C,
@@ -1051,7 +1080,7 @@ cudaError_t launch_swap(const DeviceInfo& dev, int split, int ws_split, int64_t 
 
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m, int64_t k,
                         int64_t n, const uint16_t* A, const uint16_t* B, float* C, float* workspace,
-                        cudaStream_t stream, uint64_t* launches, bool overwrite, bool bt,
+                        cudaStream_t stream, uint64_t* launches, bool overwrite, int bt,
                         const KSegments* seg) {
   // With k slices through the workspace the kernels write partial[slice][b][m][n] there (plain
   // stores) and the reduce launch below adds the slices and C.

@@ -128,10 +128,12 @@ struct KSegments {
 };
 // CTA pairs (cta_group::2) the current device can hold at once.
 int gemm_pair_units(int sms);
+// b_layout: 0 = B row-major [b][k][n], 1 = column-major [b][n][k], a multiple of 64 = packed in
+// strips of that many columns, [b][ceil(n / strip)][k][strip].
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m,
                         int64_t k, int64_t n, const uint16_t* A, const uint16_t* B, float* C,
                         float* workspace, cudaStream_t stream, uint64_t* launches,
-                        bool overwrite = false, bool b_col_major = false, const KSegments* seg = nullptr);
+                        bool overwrite = false, int b_layout = 0, const KSegments* seg = nullptr);
 
 // ---- B stored column-major where the TMA engine cannot address it ------------
 // C[b, i, j] (+)= sum_p A[b, i, p] * Bt[b, j, p]: one warp per output column, lanes stride over
@@ -139,5 +141,12 @@ cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, 
 cudaError_t colmajor_fallback_launch(int64_t b, int64_t m, int64_t k, int64_t n, const uint16_t* A,
                                      const uint16_t* Bt, float* C, bool overwrite,
                                      cudaStream_t stream, uint64_t* launches);
+
+// ---- B packed in strips where the tensor kernels cannot run --------------------
+// C[b, i, j] (+)= sum_p A[b, i, p] * Bp[b][j / strip][p][j mod strip]: one thread per output
+// element.  Any strip and shape, no alignment needs; slow, deterministic.
+cudaError_t packed_fallback_launch(int64_t strip, int64_t b, int64_t m, int64_t k, int64_t n,
+                                   const uint16_t* A, const uint16_t* Bp, float* C, bool overwrite,
+                                   cudaStream_t stream, uint64_t* launches);
 
 }  // namespace morello

@@ -536,6 +536,46 @@ cudaError_t colmajor_fallback_launch(int64_t b, int64_t m, int64_t k, int64_t n,
   return cudaSuccess;
 }
 
+namespace {
+
+// Packed B where the tensor kernels cannot run: one thread per output column and (row, batch)
+// pair taken in strides of the grid; neighbouring threads read neighbouring columns of a strip
+// (coalesced inside a strip), k in increasing order.
+__global__ void __launch_bounds__(256)
+packed_fallback_kernel(const uint16_t* __restrict__ A, const uint16_t* __restrict__ Bp,
+                       float* __restrict__ C, int64_t b, int64_t m, int64_t k, int64_t n,
+                       int64_t strip, int overwrite) {
+  const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= n) return;
+  const int64_t strips = (n + strip - 1) / strip;
+  for (int64_t bb = blockIdx.z; bb < b; bb += gridDim.z) {
+    const uint16_t* col = Bp + ((bb * strips + j / strip) * k) * strip + (j % strip);
+    for (int64_t i = blockIdx.y; i < m; i += gridDim.y) {
+      const uint16_t* arow = A + (bb * m + i) * k;
+      float sum = 0.f;
+      for (int64_t p = 0; p < k; ++p)
+        sum = fmaf(__uint_as_float(((uint32_t)arow[p]) << 16),
+                   __uint_as_float(((uint32_t)col[p * strip]) << 16), sum);
+      float* c = C + (bb * m + i) * n + j;
+      *c = overwrite ? sum : *c + sum;
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t packed_fallback_launch(int64_t strip, int64_t b, int64_t m, int64_t k, int64_t n,
+                                   const uint16_t* A, const uint16_t* Bp, float* C, bool overwrite,
+                                   cudaStream_t stream, uint64_t* launches) {
+  dim3 grid((unsigned)((n + 255) / 256), (unsigned)std::min<int64_t>(m, 65535),
+            (unsigned)std::min<int64_t>(b, 65535));
+  packed_fallback_kernel<<<grid, 256, 0, stream>>>(A, Bp, C, b, m, k, n, strip, overwrite ? 1 : 0);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  ++*launches;
+  return cudaSuccess;
+}
+
 cudaError_t skinny_reduce_launch(const float* partial, float* C, int64_t b, int m, int64_t n,
                                  int64_t c_batch, int split_k, cudaStream_t stream, bool overwrite) {
   const int64_t total = b * m * n;
