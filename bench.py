@@ -417,6 +417,42 @@ def bench_colmajor(torch, mb, idx, iters, peaks, windows):
             "frac_tensor_measured_burst": cfg.flops / sec / 1e12 / peaks["bf16_tflops"]}
 
 
+def bench_packed(torch, mb, idx, strip, iters, peaks, windows):
+    """A config with its B packed in strips of `strip` columns (Bp[b][n/strip][k][strip])
+    through morello_matmul_accum_packed_b; inputs rotate like bench_config's."""
+    cfg = w.CONFIGS[idx]
+    b, m, k, n = cfg.shape
+    in_bytes = 2 * b * m * k + 2 * b * k * n + 4 * b * m * n
+    sets = max(1, min(ROTATE, int(np.ceil(512 * 2 ** 20 / in_bytes))))
+    dev = []
+    for s_ in range(sets):
+        As, Bs, Cs = w.make(b, m, k, n, 1000 * idx + 100 * s_ + 70, cfg.ab, "zeros")
+        dev.append((torch.from_numpy(As.view(np.int16)).cuda(),
+                    torch.from_numpy(w.pack_b(Bs, strip).view(np.int16)).cuda(), torch.from_numpy(Cs).cuda()))
+    ptrs = [(a.data_ptr(), bb.data_ptr(), c.data_ptr()) for (a, bb, c) in dev]
+    stream = torch.cuda.current_stream().cuda_stream
+    call = mb.lib().morello_matmul_accum_packed_b
+
+    def step(i):
+        pa, pb, pc = ptrs[i % sets]
+        rc = call(strip, b, m, k, n, pa, pb, pc, stream)
+        if rc != 0:
+            raise mb.MorelloError(rc, "bench packed %s" % cfg.name)
+
+    l0 = mb.morello_launch_count()
+    step(0)
+    per_call = mb.morello_launch_count() - l0
+    t0 = time.perf_counter()
+    loops = [time_calls(torch, step, iters, 5 if r == 0 else 3) for r in range(3)]
+    windows.append((t0, time.perf_counter()))
+    sec = min(loops) / iters
+    return {"name": cfg.name, "op": "matmul_accum_packed_b", "strip": strip, "shape": list(cfg.shape),
+            "path": "tcgen05", "us_per_call": sec * 1e6, "GBps": cfg.algorithmic_bytes / sec / 1e9,
+            "TFLOPs": cfg.flops / sec / 1e12, "iters": iters, "launches_per_call": per_call,
+            "rotating_sets": sets, "frac_hbm_measured": cfg.algorithmic_bytes / sec / 1e9 / peaks["hbm_gbs"],
+            "frac_tensor_measured_burst": cfg.flops / sec / 1e12 / peaks["bf16_tflops"]}
+
+
 def run_case(args):
     """One configuration alone, device-timed: the command the ncu captures under
     profiles/ were taken with, and the unit of the sweeps quoted in the design notes."""
@@ -592,6 +628,8 @@ def run_ours(args):
         extra.append(bench_colmajor(torch, mb, HEADLINE, 300, peaks, windows))
         if 3 in args.configs:
             extra.append(bench_colmajor(torch, mb, 3, 30, peaks, windows))
+        if 2 in args.configs:
+            extra.append(bench_packed(torch, mb, 2, 64, 300, peaks, windows))
         for name, shape, iters, note in (
                 ("route_gemv_long_k", (1, 1, 8192, 16384), 100, "single row on the operand-swapped tensor kernel"),
                 ("route_k_slices", (1, 512, 16384, 2048), 100, "few tiles, long k: k slices through the workspace + reduce launch"),
