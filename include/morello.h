@@ -9,7 +9,8 @@
  *
  *     C[b,i,j]  <-  C[b,i,j] + sum_{p<k} A[b,i,p] * B[b,p,j]
  *
- * Layout (all entry points): dense row-major, no leading dimensions,
+ * Layout (unless an entry point says otherwise: B may also be given column-major or packed in
+ * strips of columns, A and B as float32): dense row-major, no leading dimensions,
  *     A[b][m][k]  bf16   (read only)
  *     B[b][k][n]  bf16   (read only, one matrix per batch, no broadcasting)
  *     C[b][m][n]  f32    (read-modify-write)
