@@ -469,6 +469,9 @@ struct SwapParams {
   int split_k;      // k slices per strip (cluster form: the slices of a strip are one cluster;
                     // otherwise every slice writes its own copy of the output, see the kernel)
   int kb_per_slice; // k blocks per slice
+  int strips;       // 128-column strips per batch
+  int64_t items;    // batches x strips x slices
+  int64_t bsz;      // batches
   int seg_blocks;   // > 0: k blocks per segment of the k range (see KSegments); 0: k as stored
   uint32_t seg_a, seg_b;
   int pack_strip;   // > 0: B is packed in strips of this many columns (a multiple of 64)
@@ -480,6 +483,7 @@ struct SwapBarriers {
   uint64_t full[kMaxStages];
   uint64_t empty[kMaxStages];
   uint64_t acc_full;
+  uint64_t acc_empty;
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -489,7 +493,13 @@ struct SwapBarriers {
 // (the stage ring is free by then) and the blocks share the rows out among themselves: each adds
 // its rows' slices through distributed shared memory in slice order, then C: one launch, no
 // scratch, a fixed order.
-template <int kRowsA, bool kClusterK>
+// Without a cluster the grid is persistent: a block walks the (batch, strip, slice) items
+// blockIdx.x, blockIdx.x + gridDim.x, ...; its producer keeps the stage ring full across items,
+// so the loads of the next items run under the epilogue of the current one.  With many short
+// items (batched problems with a short k) that removes the per-block set-up from the critical
+// path (256 x 1 x 128 x 4096: 71.8 us with one block per item).  With one item per block (the
+// long streams the kernel was tuned on) nothing changes.
+template <int kRowsA, bool kClusterK, bool kPersistent>
 __global__ void __launch_bounds__(kThreads)
 swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
             const SwapParams p) {
@@ -502,12 +512,31 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int strip = blockIdx.x / p.split_k;
-  const int slice = blockIdx.x % p.split_k;     // cluster form: = rank in the cluster
-  const int col0 = strip * kSwapStripCols;
-  const int bb = blockIdx.y;
-  const int kb_begin = slice * p.kb_per_slice;
-  const int kb_end = min(p.k_blocks, kb_begin + p.kb_per_slice);
+  static_assert(!(kClusterK && kPersistent), "a cluster takes one item per block");
+  // Items: one per block (blockIdx.x = strip x slice, blockIdx.y = batch: the loops below then
+  // run once and cost nothing), or, persistent, item t = (batch * strips + strip) * slices +
+  // slice walked in strides of the grid.
+  const int per_batch = p.strips * p.split_k;
+  const int first = kPersistent ? (int)blockIdx.x : 0;
+  const int stride = kPersistent ? (int)gridDim.x : 1;
+  const int last = kPersistent ? (int)p.items : first + 1;     // items [first, last) in steps of stride
+  struct Work { int bb, col0, slice, kb_begin, kb_end; };
+  auto decode = [&](int t) {
+    Work w;
+    int r;
+    if constexpr (kPersistent) {
+      w.bb = t / per_batch;
+      r = t - w.bb * per_batch;
+    } else {
+      w.bb = (int)blockIdx.y;
+      r = (int)blockIdx.x;
+    }
+    w.col0 = (r / p.split_k) * kSwapStripCols;
+    w.slice = r % p.split_k;
+    w.kb_begin = w.slice * p.kb_per_slice;
+    w.kb_end = min(p.k_blocks, w.kb_begin + p.kb_per_slice);
+    return w;
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S::kStages; ++s) {
@@ -515,18 +544,22 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       mbar_init(&bars->empty[s], 1);
     }
     mbar_init(&bars->acc_full, 1);
+    mbar_init(&bars->acc_empty, 4);     // one arrival per epilogue warp
     bars->abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_descriptor(&map_a);
     tma_prefetch_descriptor(&map_b);
-    const int ahead = min(kb_end, kb_begin + kSwapPrefetchBlocks);
-    const BBox box0 = b_box(p.bt, p.pack_strip, p.pack_strips, col0, 0, bb);
-    const BBox box1 = b_box(p.bt, p.pack_strip, p.pack_strips, col0 + 64, 0, bb);
-    for (int kb = kb_begin; kb < ahead; ++kb) {
-      const int kbb = k_coord(kb, p.seg_blocks, p.seg_b);
-      const BBox c0 = at_k(box0, p.bt, kbb), c1 = at_k(box1, p.bt, kbb);
-      tma_prefetch_l2_3d(&map_b, c0.x, c0.y, c0.z);
-      tma_prefetch_l2_3d(&map_b, c1.x, c1.y, c1.z);
+    if (first < last) {
+      const Work w = decode(first);
+      const int ahead = min(w.kb_end, w.kb_begin + kSwapPrefetchBlocks);
+      const BBox box0 = b_box(p.bt, p.pack_strip, p.pack_strips, w.col0, 0, w.bb);
+      const BBox box1 = b_box(p.bt, p.pack_strip, p.pack_strips, w.col0 + 64, 0, w.bb);
+      for (int kb = w.kb_begin; kb < ahead; ++kb) {
+        const int kbb = k_coord(kb, p.seg_blocks, p.seg_b);
+        const BBox c0 = at_k(box0, p.bt, kbb), c1 = at_k(box1, p.bt, kbb);
+        tma_prefetch_l2_3d(&map_b, c0.x, c0.y, c0.z);
+        tma_prefetch_l2_3d(&map_b, c1.x, c1.y, c1.z);
+      }
     }
   }
   if (warp == 1) {
@@ -547,19 +580,23 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     if (elect_one()) {
       int stage = 0;
       uint32_t phase = 0;
-      const BBox box0 = b_box(p.bt, p.pack_strip, p.pack_strips, col0, 0, bb);
-      const BBox box1 = b_box(p.bt, p.pack_strip, p.pack_strips, col0 + 64, 0, bb);
-      for (int kb = kb_begin; kb < kb_end; ++kb) {
-        if (!mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag, p.status, 8)) break;
-        uint8_t* sb = stages + (size_t)stage * S::kStageBytes;
-        uint8_t* sa = sb + S::kBytesStrip;
-        mbar_arrive_expect_tx(&bars->full[stage], S::kStageBytes);
-        const int ka = k_coord(kb, p.seg_blocks, p.seg_a), kbb = k_coord(kb, p.seg_blocks, p.seg_b);
-        const BBox c0 = at_k(box0, p.bt, kbb), c1 = at_k(box1, p.bt, kbb);
-        tma_load_3d(sb, &map_b, &bars->full[stage], c0.x, c0.y, c0.z);
-        tma_load_3d(sb + kBoxBytesB, &map_b, &bars->full[stage], c1.x, c1.y, c1.z);
-        tma_load_3d(sa, &map_a, &bars->full[stage], ka, 0, bb);
-        if (++stage == S::kStages) { stage = 0; phase ^= 1; }
+      bool ok = true;
+      for (int t = first; t < last && ok; t += stride) {
+        const Work w = decode(t);
+        const BBox box0 = b_box(p.bt, p.pack_strip, p.pack_strips, w.col0, 0, w.bb);
+        const BBox box1 = b_box(p.bt, p.pack_strip, p.pack_strips, w.col0 + 64, 0, w.bb);
+        for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
+          if (!(ok = mbar_wait(&bars->empty[stage], phase ^ 1, abort_flag, p.status, 8))) break;
+          uint8_t* sb = stages + (size_t)stage * S::kStageBytes;
+          uint8_t* sa = sb + S::kBytesStrip;
+          mbar_arrive_expect_tx(&bars->full[stage], S::kStageBytes);
+          const int ka = k_coord(kb, p.seg_blocks, p.seg_a), kbb = k_coord(kb, p.seg_blocks, p.seg_b);
+          const BBox c0 = at_k(box0, p.bt, kbb), c1 = at_k(box1, p.bt, kbb);
+          tma_load_3d(sb, &map_b, &bars->full[stage], c0.x, c0.y, c0.z);
+          tma_load_3d(sb + kBoxBytesB, &map_b, &bars->full[stage], c1.x, c1.y, c1.z);
+          tma_load_3d(sa, &map_a, &bars->full[stage], ka, 0, w.bb);
+          if (++stage == S::kStages) { stage = 0; phase ^= 1; }
+        }
       }
       // Every load of this block is in flight: the next kernel's blocks may come in.
       pdl_release();
@@ -572,86 +609,110 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       const uint32_t idesc = p.bt ? instr_desc_bf16(kSwapStripCols, kRowsA, false, false)
                                   : instr_desc_bf16(kSwapStripCols, kRowsA, true, false);
       int stage = 0;
-      uint32_t phase = 0;
+      uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int kb = kb_begin; kb < kb_end; ++kb) {
-        if (!(ok = mbar_wait(&bars->full[stage], phase, abort_flag, p.status, 9))) break;
-        tc_fence_after_sync();
-        const uint32_t sb = smem_u32(stages + (size_t)stage * S::kStageBytes);
-        const uint32_t sa = sb + S::kBytesStrip;
-#pragma unroll
-        for (int j = 0; j < kTileK / 16; ++j) {
-          // The strip of B: 64-column groups one TMA box apart, 8-row k groups 1024 bytes
-          // apart, 16 k rows = 2048 bytes.  The rows of A: 8-row groups 1024 bytes apart,
-          // 16 k elements = 32 bytes along the row.
-          const uint64_t d_strip = p.bt ? smem_desc_sw128(sb + j * 32, 16, 1024)
-                                        : smem_desc_sw128(sb + j * 2048, kBoxBytesB, 1024);
-          const uint64_t d_rows = smem_desc_sw128(sa + j * 32, 16, 1024);
-          mma_bf16_ss(tmem_base, d_strip, d_rows, idesc, ((kb - kb_begin) | j) != 0 ? 1u : 0u);
+      for (int t = first; t < last && ok; t += stride) {
+        const Work w = decode(t);
+        // The epilogue has read the previous item's sums out of the accumulator.
+        if constexpr (kPersistent) {
+          if (!(ok = mbar_wait(&bars->acc_empty, acc_phase ^ 1, abort_flag, p.status, 11))) break;
+          tc_fence_after_sync();
         }
-        mma_commit(&bars->empty[stage]);
-        if (++stage == S::kStages) { stage = 0; phase ^= 1; }
+        for (int kb = w.kb_begin; kb < w.kb_end; ++kb) {
+          if (!(ok = mbar_wait(&bars->full[stage], phase, abort_flag, p.status, 9))) break;
+          tc_fence_after_sync();
+          const uint32_t sb = smem_u32(stages + (size_t)stage * S::kStageBytes);
+          const uint32_t sa = sb + S::kBytesStrip;
+#pragma unroll
+          for (int j = 0; j < kTileK / 16; ++j) {
+            // The strip of B: 64-column groups one TMA box apart, 8-row k groups 1024 bytes
+            // apart, 16 k rows = 2048 bytes.  The rows of A: 8-row groups 1024 bytes apart,
+            // 16 k elements = 32 bytes along the row.
+            const uint64_t d_strip = p.bt ? smem_desc_sw128(sb + j * 32, 16, 1024)
+                                          : smem_desc_sw128(sb + j * 2048, kBoxBytesB, 1024);
+            const uint64_t d_rows = smem_desc_sw128(sa + j * 32, 16, 1024);
+            mma_bf16_ss(tmem_base, d_strip, d_rows, idesc, ((kb - w.kb_begin) | j) != 0 ? 1u : 0u);
+          }
+          mma_commit(&bars->empty[stage]);
+          if (++stage == S::kStages) { stage = 0; phase ^= 1; }
+        }
+        if (ok) mma_commit(&bars->acc_full);
+        acc_phase ^= 1;
       }
-      if (ok) mma_commit(&bars->acc_full);
     }
   } else {
     // ------------------------------------------------------------------ epilogue
     const int quarter = warp & 3;  // TMEM lanes [32 * quarter, 32 * quarter + 32)
-    const int64_t col = (int64_t)col0 + quarter * 32 + lane;   // this thread's column of C
-    const bool col_live = col < p.n;
-    // Without a cluster, slices > 1 means that C is partial[slice][b][m][n] in the workspace.
-    const int64_t out_b = kClusterK ? bb : (int64_t)slice * gridDim.y + bb;
-    float* c_col = p.C + out_b * p.c_batch + col;
-    // Cluster form: block r of the cluster finishes the rows i with i % split_k == r.
-    float c_in[kRowsA];
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int t = first; t < last; t += stride) {
+      const Work w = decode(t);
+      const int slice = w.slice;
+      const int64_t col = (int64_t)w.col0 + quarter * 32 + lane;   // this thread's column of C
+      const bool col_live = col < p.n;
+      // Without a cluster, slices > 1 means that C is partial[slice][b][m][n] in the workspace.
+      const int64_t out_b = kClusterK ? w.bb : (int64_t)slice * p.bsz + w.bb;
+      float* c_col = p.C + out_b * p.c_batch + col;
+      // Cluster form: block r of the cluster finishes the rows i with i % split_k == r.
+      float c_in[kRowsA];
 #pragma unroll
-    for (int i = 0; i < kRowsA; ++i) {
-      const bool mine = !kClusterK || (i % p.split_k) == slice;
-      c_in[i] = (mine && col_live && i < p.m && !p.overwrite) ? c_col[(int64_t)i * p.n] : 0.f;
-    }
-    bool ok = mbar_wait(&bars->acc_full, 0, abort_flag, p.status, 10);
-    ok = __all_sync(0xffffffffu, ok);  // also reconverges the warp for the aligned TMEM loads
-    if (ok) {
-      tc_fence_after_sync();
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-      // Cluster form: every MMA has completed, so the stage ring is free; the accumulator is
-      // parked there as part[row][128 columns of the strip].
-      float* part = reinterpret_cast<float*>(stages);
+      for (int i = 0; i < kRowsA; ++i) {
+        const bool mine = !kClusterK || (i % p.split_k) == slice;
+        c_in[i] = (mine && col_live && i < p.m && !p.overwrite) ? c_col[(int64_t)i * p.n] : 0.f;
+      }
+      if (ok) ok = mbar_wait(&bars->acc_full, acc_phase, abort_flag, p.status, 10);
+      ok = __all_sync(0xffffffffu, ok);  // also reconverges the warp for the aligned TMEM loads
+      acc_phase ^= 1;
+      if (ok) {
+        tc_fence_after_sync();
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        // Cluster form: every MMA has completed, so the stage ring is free; the accumulator is
+        // parked there as part[row][128 columns of the strip].
+        float* part = reinterpret_cast<float*>(stages);
 #pragma unroll
-      for (int g = 0; g < kRowsA / 16; ++g) {
-        uint32_t r[16];
-        tmem_ld_32x16(taddr + g * 16, r);
-        tmem_ld_wait();
+        for (int g = 0; g < kRowsA / 16; ++g) {
+          uint32_t r[16];
+          tmem_ld_32x16(taddr + g * 16, r);
+          tmem_ld_wait();
+          if (kPersistent && g == kRowsA / 16 - 1) {
+            // The last of the sums is in registers: the MMA warp may start the next item.
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->acc_empty);
+          }
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          if constexpr (kClusterK) {
-            part[(g * 16 + i) * kSwapStripCols + quarter * 32 + lane] = __uint_as_float(r[i]);
-          } else {
-            if (col_live && g * 16 + i < p.m)
-              c_col[(int64_t)(g * 16 + i) * p.n] = c_in[g * 16 + i] + __uint_as_float(r[i]);
+          for (int i = 0; i < 16; ++i) {
+            if constexpr (kClusterK) {
+              part[(g * 16 + i) * kSwapStripCols + quarter * 32 + lane] = __uint_as_float(r[i]);
+            } else {
+              if (col_live && g * 16 + i < p.m)
+                c_col[(int64_t)(g * 16 + i) * p.n] = c_in[g * 16 + i] + __uint_as_float(r[i]);
+            }
           }
         }
+      } else if (!kClusterK) {
+        break;      // timed out: nothing more is written (the cluster form still meets its barriers)
       }
-    }
-    if constexpr (kClusterK) {
-      // Both cluster barriers are executed by every thread of every block (see below); between
-      // them every block finishes its share of the rows: the slices' sums in slice order (read
-      // through distributed shared memory), then C, then the store.
-      __syncwarp();
-      cluster_sync();
-      if (!*abort_flag) {
-        const float* part = reinterpret_cast<const float*>(stages);
+      if constexpr (kClusterK) {
+        // Both cluster barriers are executed by every thread of every block (see below); between
+        // them every block finishes its share of the rows: the slices' sums in slice order (read
+        // through distributed shared memory), then C, then the store.
+        __syncwarp();
+        cluster_sync();
+        if (!*abort_flag) {
+          const float* part = reinterpret_cast<const float*>(stages);
 #pragma unroll
-        for (int i = 0; i < kRowsA; ++i) {
-          if (!col_live || i >= p.m || (i % p.split_k) != slice) continue;
-          const float* mine = part + i * kSwapStripCols + quarter * 32 + lane;
-          float sum = *peer_shared(mine, 0u);
-          for (int s2 = 1; s2 < p.split_k; ++s2) sum += *peer_shared(mine, (uint32_t)s2);
-          c_col[(int64_t)i * p.n] = c_in[i] + sum;
+          for (int i = 0; i < kRowsA; ++i) {
+            if (!col_live || i >= p.m || (i % p.split_k) != slice) continue;
+            const float* mine = part + i * kSwapStripCols + quarter * 32 + lane;
+            float sum = *peer_shared(mine, 0u);
+            for (int s2 = 1; s2 < p.split_k; ++s2) sum += *peer_shared(mine, (uint32_t)s2);
+            c_col[(int64_t)i * p.n] = c_in[i] + sum;
+          }
         }
+        __syncwarp();
+        cluster_sync();
       }
-      __syncwarp();
-      cluster_sync();
     }
   }
   if constexpr (kClusterK) {
@@ -875,10 +936,10 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob
   // 4096: 14.4 / 16.0).  Beyond 64 rows the 128-row tiles win: an accumulator of more than 64
   // columns per thread cannot be paired with an early read of C in registers, and sending the
   // sums out as L2 reductions instead cost more than it saved (96 rows: 16.7 against 15.4 us).
-  if (form == 3 || (form == 0 && tile_n == 0 && m <= kSwapMaxRows && b <= 65535)) {
+  if (form == 3 || (form == 0 && tile_n == 0 && m <= kSwapMaxRows)) {
     // With form 3 the knob's column field is the number of k slices instead (0 = by shape).
     const int forced_split = tile_n / 64;
-    if (m > kSwapMaxRows || b > 65535 ||
+    if (m > kSwapMaxRows || (b > 65535 && forced_split > 1) ||
         (forced_split != 0 && forced_split != 1 && forced_split != 2 && forced_split != 4 && forced_split != 8))
       return GemmPlan{false, 0, 0, 0, false, 1, 1};
     const int64_t strips = b * ((n + kSwapStripCols - 1) / kSwapStripCols);
@@ -891,7 +952,7 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob
       // strips: 14.2 / 24.1 / 19.3).  So: up to 16 rows and up to 32 strips, as many slices as
       // leave four k blocks each; the other shapes of few strips go through the workspace.
       split = 1;
-      if (forced_ws <= 1 && a_box_rows(m) == 16 && strips <= 32)
+      if (forced_ws <= 1 && a_box_rows(m) == 16 && strips <= 32 && b <= 65535)
         while (split < 8 && k_blocks >= 8 * split) split *= 2;
     }
     while (split > 1 && (k_blocks + split - 1) / split * (split - 1) >= k_blocks) split /= 2;   // no empty slice
@@ -1014,7 +1075,11 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
 
 namespace {
 
-template <int kRowsA, bool kClusterK>
+// Blocks of the operand-swapped kernel the device holds at once: two per SM with the small ring.
+template <int kRowsA>
+int64_t swap_resident(int sms) { return (int64_t)sms * (kRowsA <= 16 ? 2 : 1); }
+
+template <int kRowsA, bool kClusterK, bool kPersistent>
 cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_t m, int64_t k, int64_t n,
                              const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
                              bool overwrite, int bt, const KSegments* seg, cudaStream_t stream) {
@@ -1022,7 +1087,7 @@ cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(swap_kernel<kRowsA, kClusterK>,
+    attr_err = cudaFuncSetAttribute(swap_kernel<kRowsA, kClusterK, kPersistent>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::kSmemBytes);
   });
   if (attr_err != cudaSuccess) return attr_err;
@@ -1035,16 +1100,27 @@ cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_
   p.c_batch = m * n;
   p.k_blocks = (int)((k + kTileK - 1) / kTileK);
   p.split_k = std::max(1, split);
+  p.bsz = b;
   p.kb_per_slice = (p.k_blocks + p.split_k - 1) / p.split_k;
   p.status = dev.status;
   if (seg) { p.seg_blocks = seg->blocks; p.seg_a = seg->a_terms; p.seg_b = seg->b_terms; }
   const int64_t strips = (n + kSwapStripCols - 1) / kSwapStripCols;
-  // grid.y carries the batch index (the planner keeps batches beyond a grid dimension off
-  // this kernel).
-  if (b > 65535) return cudaErrorInvalidValue;
+  // Cluster form: grid.y carries the batch index (the planner keeps batches beyond a grid
+  // dimension off this kernel).
+  if ((!kPersistent && b > 65535) || strips * p.split_k >= (1ll << 31)) return cudaErrorInvalidValue;
   p.C = C;
+  p.strips = (int)strips;
+  p.items = b * strips * p.split_k;
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3((unsigned)(strips * p.split_k), (unsigned)b, 1);
+  if (!kPersistent) {
+    cfg.gridDim = dim3((unsigned)(strips * p.split_k), (unsigned)b, 1);
+  } else {
+    // Persistent: the items shared out evenly among as many blocks as fit the device at once.
+    if (p.items >= (1ll << 31)) return cudaErrorInvalidValue;
+    const int64_t resident = swap_resident<kRowsA>(dev.sms);
+    const int64_t per_block = (p.items + resident - 1) / resident;
+    cfg.gridDim = dim3((unsigned)((p.items + per_block - 1) / per_block), 1, 1);
+  }
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = S::kSmemBytes;
   cfg.stream = stream;
@@ -1061,7 +1137,7 @@ cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_
   }
   cfg.attrs = attr;
   cfg.numAttrs = num_attrs;
-  return cudaLaunchKernelEx(&cfg, swap_kernel<kRowsA, kClusterK>, map_a, map_b, p);
+  return cudaLaunchKernelEx(&cfg, swap_kernel<kRowsA, kClusterK, kPersistent>, map_a, map_b, p);
 }
 
 // `split` > 1: the slices of a strip form a cluster and C is the output.  `ws_split` > 1: the
@@ -1070,10 +1146,16 @@ template <int kRowsA>
 cudaError_t launch_swap(const DeviceInfo& dev, int split, int ws_split, int64_t b, int64_t m, int64_t k,
                         int64_t n, const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
                         bool overwrite, int bt, const KSegments* seg, cudaStream_t stream) {
-  return split > 1 ? launch_swap_form<kRowsA, true>(dev, split, b, m, k, n, map_a, map_b, C, overwrite,
-                                                    bt, seg, stream)
-                   : launch_swap_form<kRowsA, false>(dev, ws_split, b, m, k, n, map_a, map_b, C,
-                                                     overwrite, bt, seg, stream);
+  if (split > 1)
+    return launch_swap_form<kRowsA, true, false>(dev, split, b, m, k, n, map_a, map_b, C, overwrite, bt, seg,
+                                                 stream);
+  // More items than blocks fit at once (and batches beyond a grid dimension): persistent.
+  const int64_t items = b * ((n + kSwapStripCols - 1) / kSwapStripCols) * std::max(1, ws_split);
+  if (items > swap_resident<kRowsA>(dev.sms) || b > 65535)
+    return launch_swap_form<kRowsA, false, true>(dev, ws_split, b, m, k, n, map_a, map_b, C, overwrite, bt,
+                                                 seg, stream);
+  return launch_swap_form<kRowsA, false, false>(dev, ws_split, b, m, k, n, map_a, map_b, C, overwrite, bt,
+                                                seg, stream);
 }
 
 }  // namespace

@@ -277,3 +277,29 @@ def test_k_slices_with_matmul_and_a_caller_workspace():
     mb.morello_matmul_forced(TC, knob, b, m, k, n, dA, dB, dC, 0, 0)
     torch.cuda.synchronize()
     assert_bit_exact(dC.cpu().numpy(), oracle.matmul_accum(b, m, k, n, A, B, np.zeros_like(C)), "matmul, slices")
+
+
+# ------------------------------------------------ operand-swapped kernel, persistent form
+@pytest.mark.parametrize("shape", [
+    (256, 1, 128, 4096),     # 8,192 items of two k blocks on 296 blocks
+    (700, 3, 72, 264),       # ragged k block, ragged strip, items not a multiple of the blocks
+    (40, 33, 200, 1000),     # 48-row instantiation: one block per SM
+    (66000, 2, 64, 128),     # more batches than a grid dimension
+    (3, 16, 4096, 16384),    # long items: 384 items of 64 k blocks
+])
+def test_swap_form_persistent_blocks_walk_many_items(shape):
+    b, m, k, n = shape
+    A, B, C = w.make(b, m, k, n, seed=sum(shape) % 997, ab="int4", c="normal")
+    got = check_full(A, B, C, integer=True, path=TC, split_k=SWAP, what="persistent %s" % (shape,))
+    assert np.array_equal(bits(gpu_run(A, B, C, path=TC, split_k=SWAP)), bits(got))
+    if b * m * k * n < 3e8:
+        A, B, C = w.make(b, m, k, n, seed=sum(shape) % 997 + 1, ab="normal_rsqrtk", c="normal")
+        check_full(A, B, C, integer=False, path=TC, split_k=SWAP, what="persistent %s random" % (shape,))
+
+
+def test_swap_form_persistent_with_k_slices_through_the_workspace():
+    b, m, k, n = 9, 40, 4096, 520            # 45 strips x 4 slices = 180 items on 148 one-per-SM blocks
+    A, B, C = w.make(b, m, k, n, seed=17, ab="int4", c="normal")
+    knob = SWAP + 16 + WS * 4
+    got = check_full(A, B, C, integer=True, path=TC, split_k=knob, what="persistent, 4 slices")
+    assert_bit_exact(gpu_run(A, B, C, path=TC, split_k=SWAP + 16 + WS), got, "slices vs whole k")
