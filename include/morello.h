@@ -264,6 +264,17 @@ size_t morello_workspace_bytes_forced(int path, int split_k,
 int morello_read_device_status(void* stream, uint32_t* detail);
 
 /*
+ * Self-test of the bounded device-side waits (every mbarrier wait in the kernels gives up
+ * after a time limit -- 2 s in the kernels proper -- records where in the status word and lets
+ * its block return, so a stalled pipeline becomes an error code, not a hung device).  Launches
+ * one thread that waits at most `limit_ms` (1 .. 1000) on a barrier that nothing arrives on,
+ * and synchronises `stream`.  Returns MORELLO_OK when the wait gave up as designed (the status
+ * word is then set: the next morello_read_device_status returns MORELLO_ERR_DEVICE_TIMEOUT and
+ * clears it), MORELLO_ERR_CUDA if it did not.  Faults and hangs nothing.
+ */
+int morello_selftest_wait_timeout(uint32_t limit_ms, void* stream);
+
+/*
  * What the kernels size their grids by on the current device: the number of SMs and
  * the number of two-CTA clusters (cta_group::2 pairs) the device can hold at once,
  * which may be fewer than half the SMs.  Either pointer may be NULL.

@@ -40,6 +40,7 @@ SIGNATURES = {
     "morello_matmul_accum_f32": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
     "morello_matmul_accum_colmajor_b": (_int, [_int, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
     "morello_matmul_accum_packed_b": (_int, [_int, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
+    "morello_selftest_wait_timeout": (_int, [ctypes.c_uint32, _vp]),
     "morello_workspace_bytes": (_sz, [_i64, _i64, _i64, _i64]),
     "morello_matmul_accum_ws": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _sz, _vp]),
     "morello_matmul_accum_host": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp]),
@@ -193,6 +194,12 @@ def morello_matmul_accum_forced(path, split_k, b, m, k, n, A, B, C, workspace=No
 
 def morello_workspace_bytes_forced(path, split_k, b, m, k, n) -> int:
     return int(lib().morello_workspace_bytes_forced(path, split_k, b, m, k, n))
+
+
+def morello_selftest_wait_timeout(limit_ms, stream=None) -> None:
+    """Makes one bounded device-side wait run out on purpose (see the header); raises unless it
+    gave up as designed.  The device status word is set afterwards."""
+    _check(lib().morello_selftest_wait_timeout(limit_ms, _stream(stream)), "morello_selftest_wait_timeout")
 
 
 def morello_read_device_status(stream=None):

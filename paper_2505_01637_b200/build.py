@@ -13,7 +13,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmorello.so")
-SOURCES = ["api.cu", "skinny.cu", "gemv_stream.cu", "gemm_tcgen05.cu", "f32_split.cu", "pad.cu", "tensormap.cu", "noalloc.cu"]
+SOURCES = ["api.cu", "skinny.cu", "gemv_stream.cu", "gemm_tcgen05.cu", "f32_split.cu", "pad.cu", "selftest.cu", "tensormap.cu", "noalloc.cu"]
 HEADERS = [os.path.join(CSRC, "internal.h"), os.path.join(CSRC, "sm100.cuh"),
            os.path.join(CSRC, "tensormap.h"),
            os.path.join(os.path.dirname(HERE), "include", "morello.h")]

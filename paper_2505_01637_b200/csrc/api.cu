@@ -576,6 +576,29 @@ int morello_read_device_status(void* stream, uint32_t* detail) {
   return MORELLO_ERR_DEVICE_TIMEOUT;
 }
 
+int morello_selftest_wait_timeout(uint32_t limit_ms, void* stream) {
+  if (limit_ms == 0 || limit_ms > 1000) return MORELLO_ERR_INVALID_SHAPE;
+  DeviceState* st = nullptr;
+  int rc;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    rc = device_state(&st);
+  }
+  if (rc != MORELLO_OK) return rc;
+  // The second word of the status block receives the kernel's own verdict.
+  int* gave_up = reinterpret_cast<int*>(st->info.status + 1);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemsetAsync(gave_up, 0, 4, s);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = wait_timeout_selftest_launch(st->info.status, (uint64_t)limit_ms * 1000000ull, gave_up, s);
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e);
+  int verdict = 0;
+  if ((e = cudaMemcpy(&verdict, gave_up, 4, cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(e);
+  return verdict == 1 ? MORELLO_OK : MORELLO_ERR_CUDA;
+}
+
 int morello_device_limits(int* sms, int* cta_pairs) {
   DeviceState* st = nullptr;
   int rc;

@@ -149,4 +149,10 @@ cudaError_t packed_fallback_launch(int64_t strip, int64_t b, int64_t m, int64_t 
                                    const uint16_t* A, const uint16_t* Bp, float* C, bool overwrite,
                                    cudaStream_t stream, uint64_t* launches);
 
+// ---- self-test of the bounded device-side waits --------------------------------
+// One thread waits at most limit_ns on a barrier nothing arrives on, gives up, records the
+// site in `status` and sets *gave_up (device memory) to 1.
+cudaError_t wait_timeout_selftest_launch(uint32_t* status, uint64_t limit_ns, int* gave_up,
+                                         cudaStream_t stream);
+
 }  // namespace morello
