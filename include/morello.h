@@ -145,6 +145,13 @@ int morello_matmul_accum_colmajor_b(int tile, int64_t b, int64_t m, int64_t k, i
 int morello_matmul_accum_packed_b(int strip, int64_t b, int64_t m, int64_t k, int64_t n,
                                   const void* A, const void* Bp, float* C, void* stream);
 
+/* Matmul (C = A x B, C never read; k == 0 sets C to zero) with B column-major or packed:
+ * arguments, kernels and status codes as the two accumulating entry points above. */
+int morello_matmul_colmajor_b(int tile, int64_t b, int64_t m, int64_t k, int64_t n,
+                              const void* A, const void* Bt, float* C, void* stream);
+int morello_matmul_packed_b(int strip, int64_t b, int64_t m, int64_t k, int64_t n,
+                            const void* A, const void* Bp, float* C, void* stream);
+
 /*
  * MatmulAccum on float32 inputs (the paper's other benchmark, Section 7, is a float32
  * 2048-square matrix multiplication): A[b][m][k], B[b][k][n] and C[b][m][n] all f32, dense

@@ -41,6 +41,8 @@ SIGNATURES = {
     "morello_matmul_accum_colmajor_b": (_int, [_int, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
     "morello_matmul_accum_packed_b": (_int, [_int, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
     "morello_selftest_wait_timeout": (_int, [ctypes.c_uint32, _vp]),
+    "morello_matmul_colmajor_b": (_int, [_int, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
+    "morello_matmul_packed_b": (_int, [_int, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
     "morello_workspace_bytes": (_sz, [_i64, _i64, _i64, _i64]),
     "morello_matmul_accum_ws": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _sz, _vp]),
     "morello_matmul_accum_host": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp]),
@@ -152,6 +154,18 @@ def morello_matmul_accum_packed_b(strip, b, m, k, n, A, Bp, C, stream=None) -> N
     _check(lib().morello_matmul_accum_packed_b(strip, b, m, k, n, _addr(A), _addr(Bp), _addr(C),
                                                _stream(stream)),
            "morello_matmul_accum_packed_b")
+
+
+def morello_matmul_colmajor_b(tile, b, m, k, n, A, Bt, C, stream=None) -> None:
+    """C = A x B with B given column-major (C is not read)."""
+    _check(lib().morello_matmul_colmajor_b(tile, b, m, k, n, _addr(A), _addr(Bt), _addr(C), _stream(stream)),
+           "morello_matmul_colmajor_b")
+
+
+def morello_matmul_packed_b(strip, b, m, k, n, A, Bp, C, stream=None) -> None:
+    """C = A x B with B packed in strips of `strip` columns (C is not read)."""
+    _check(lib().morello_matmul_packed_b(strip, b, m, k, n, _addr(A), _addr(Bp), _addr(C), _stream(stream)),
+           "morello_matmul_packed_b")
 
 
 def morello_workspace_bytes(b, m, k, n) -> int:

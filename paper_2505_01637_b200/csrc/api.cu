@@ -431,6 +431,22 @@ int morello_matmul_accum_packed_b(int strip, int64_t b, int64_t m, int64_t k, in
   return run(MORELLO_PATH_AUTO, 0, b, m, k, n, A, Bp, C, nullptr, 0, true, stream, false, strip);
 }
 
+int morello_matmul_colmajor_b(int tile, int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
+                              const void* Bt, float* C, void* stream) {
+  if (tile < 0) return MORELLO_ERR_INVALID_SHAPE;
+  return run(MORELLO_PATH_AUTO, tile, b, m, k, n, A, Bt, C, nullptr, 0, true, stream, true, 1);
+}
+
+int morello_matmul_packed_b(int strip, int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
+                            const void* Bp, float* C, void* stream) {
+  if (strip < 1) return MORELLO_ERR_INVALID_SHAPE;
+  int64_t t;
+  if (n > 0 && (mul_overflows((n + strip - 1) / strip, strip, &t) || mul_overflows(t, k > 0 ? k : 1, &t) ||
+                mul_overflows(t, b > 0 ? b : 1, &t) || mul_overflows(t, 2, &t)))
+    return MORELLO_ERR_INVALID_SHAPE;
+  return run(MORELLO_PATH_AUTO, 0, b, m, k, n, A, Bp, C, nullptr, 0, true, stream, true, strip);
+}
+
 int morello_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n, const float* A,
                              const float* B, float* C, void* stream) {
   if (b < 0 || m < 0 || k < 0 || n < 0) return MORELLO_ERR_INVALID_SHAPE;

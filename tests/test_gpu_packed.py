@@ -93,3 +93,22 @@ def test_packed_b_bad_strip_and_empty_shapes():
     mb.morello_matmul_accum_packed_b(64, 1, 2, 0, 8, d, d, c)     # empty sum: C untouched
     torch.cuda.synchronize()
     assert float(c.min()) == 3.0 and float(c.max()) == 3.0
+
+
+@pytest.mark.parametrize("shape", [(1, 16, 520, 776), (2, 300, 1000, 328), (1, 5, 33, 50), (1, 8, 4096, 256)])
+def test_matmul_with_b_column_major_or_packed_never_reads_c(shape):
+    import torch
+    b, m, k, n = shape
+    A, B, C = w.make(b, m, k, n, seed=sum(shape), ab="int4", c="normal")
+    want = oracle.matmul_accum(b, m, k, n, A, B, np.zeros_like(C))
+    poison = np.full_like(C, np.nan)
+    dA, dBp, dC = to_dev(A, w.pack_b(B, 64, fill=NAN), poison)
+    mb.morello_matmul_packed_b(64, b, m, k, n, dA, dBp, dC)
+    torch.cuda.synchronize()
+    assert_bit_exact(dC.cpu().numpy(), want, "matmul, packed B %s" % (shape,))
+    dA, dBt, dC = to_dev(A, np.ascontiguousarray(np.swapaxes(B, 1, 2)), poison)
+    mb.morello_matmul_colmajor_b(0, b, m, k, n, dA, dBt, dC)
+    torch.cuda.synchronize()
+    assert_bit_exact(dC.cpu().numpy(), want, "matmul, column-major B %s" % (shape,))
+    st, detail = mb.morello_read_device_status()
+    assert st == mb.MORELLO_OK, hex(detail)
