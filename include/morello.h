@@ -169,6 +169,11 @@ int morello_matmul_packed_b(int strip, int64_t b, int64_t m, int64_t k, int64_t 
 int morello_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n,
                              const float* A, const float* B, float* C, void* stream);
 
+/* Matmul on float32 inputs: C = A x B, C never read (k == 0 sets C to zero); otherwise as
+ * morello_matmul_accum_f32. */
+int morello_matmul_f32(int64_t b, int64_t m, int64_t k, int64_t n,
+                       const float* A, const float* B, float* C, void* stream);
+
 /*
  * End-to-end convenience call on HOST buffers (same layouts): copies A, B and
  * C to library-owned device staging (grown on demand), runs the operation,

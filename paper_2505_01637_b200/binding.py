@@ -38,6 +38,7 @@ SIGNATURES = {
     "morello_matmul_forced": (_int, [_int, _int, _i64, _i64, _i64, _i64, _vp, _vp, _vp,
                                      _vp, _sz, _vp]),
     "morello_matmul_accum_f32": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
+    "morello_matmul_f32": (_int, [_i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
     "morello_matmul_accum_colmajor_b": (_int, [_int, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
     "morello_matmul_accum_packed_b": (_int, [_int, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
     "morello_selftest_wait_timeout": (_int, [ctypes.c_uint32, _vp]),
@@ -140,6 +141,12 @@ def morello_matmul_accum_f32(b, m, k, n, A, B, C, stream=None) -> None:
     """C += A x B with float32 A and B (split into bf16 terms inside the library)."""
     _check(lib().morello_matmul_accum_f32(b, m, k, n, _addr(A), _addr(B), _addr(C), _stream(stream)),
            "morello_matmul_accum_f32")
+
+
+def morello_matmul_f32(b, m, k, n, A, B, C, stream=None) -> None:
+    """C = A x B with float32 A and B (C is not read)."""
+    _check(lib().morello_matmul_f32(b, m, k, n, _addr(A), _addr(B), _addr(C), _stream(stream)),
+           "morello_matmul_f32")
 
 
 def morello_matmul_accum_colmajor_b(tile, b, m, k, n, A, Bt, C, stream=None) -> None:

@@ -447,8 +447,16 @@ int morello_matmul_packed_b(int strip, int64_t b, int64_t m, int64_t k, int64_t 
   return run(MORELLO_PATH_AUTO, 0, b, m, k, n, A, Bp, C, nullptr, 0, true, stream, true, strip);
 }
 
-int morello_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n, const float* A,
-                             const float* B, float* C, void* stream) {
+#pragma GCC visibility pop
+}  // extern "C"
+
+namespace morello {
+namespace {
+
+// Float32 inputs: split into bf16 terms, then the bf16 problem (accumulating, or, `overwrite`,
+// C = A x B with C never read).
+int run_f32(int64_t b, int64_t m, int64_t k, int64_t n, const float* A, const float* B, float* C,
+            void* stream, bool overwrite) {
   if (b < 0 || m < 0 || k < 0 || n < 0) return MORELLO_ERR_INVALID_SHAPE;
   int64_t k6, t;
   if (mul_overflows(k, 6, &k6) || mul_overflows(m, k6, &t) || mul_overflows(b, t, &t) ||
@@ -467,7 +475,9 @@ int morello_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n, const f
     std::lock_guard<std::mutex> lock(g_mutex);
     rc = device_state(&st);
   }
-  if (rc != MORELLO_OK || empty) return rc;
+  if (rc != MORELLO_OK) return rc;
+  if (empty)   // an empty sum: the bf16 path knows what that means for either operation
+    return run(MORELLO_PATH_AUTO, 0, b, m, k6, n, A, B, C, nullptr, 0, true, stream, overwrite);
   const size_t need = f32_split_bytes(b, m, k, n);
   {
     std::lock_guard<std::mutex> lock(g_mutex);
@@ -497,13 +507,29 @@ int morello_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n, const f
                                          static_cast<cudaStream_t>(stream), &launches);
   g_launches.fetch_add(launches, std::memory_order_relaxed);
   if (e != cudaSuccess) return cuda_fail(e);
-  if (!three) return run(MORELLO_PATH_AUTO, 0, b, m, k6, n, A6, B6, C, nullptr, 0, true, stream);
+  if (!three) return run(MORELLO_PATH_AUTO, 0, b, m, k6, n, A6, B6, C, nullptr, 0, true, stream, overwrite);
   // Six segments of k / 64 blocks; stored terms 0, 1, 2 = first, second, third bf16 term.
   // A: 3, 1, 2, 2, 1, 1 and B: 1, 3, 2, 1, 2, 1 (smallest products first), three bits each.
   const KSegments seg{(int)(k / 64),
                       2u | (0u << 3) | (1u << 6) | (1u << 9) | (0u << 12) | (0u << 15),
                       0u | (2u << 3) | (1u << 6) | (0u << 9) | (1u << 12) | (0u << 15), 3 * k};
-  return run(MORELLO_PATH_TCGEN05, 0, b, m, k6, n, A6, B6, C, nullptr, 0, true, stream, false, 0, &seg);
+  return run(MORELLO_PATH_TCGEN05, 0, b, m, k6, n, A6, B6, C, nullptr, 0, true, stream, overwrite, 0, &seg);
+}
+
+}  // namespace
+}  // namespace morello
+
+#pragma GCC visibility push(default)
+extern "C" {
+
+int morello_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n, const float* A,
+                             const float* B, float* C, void* stream) {
+  return run_f32(b, m, k, n, A, B, C, stream, false);
+}
+
+int morello_matmul_f32(int64_t b, int64_t m, int64_t k, int64_t n, const float* A, const float* B,
+                       float* C, void* stream) {
+  return run_f32(b, m, k, n, A, B, C, stream, true);
 }
 
 int morello_matmul_accum_host(int64_t b, int64_t m, int64_t k, int64_t n, const void* A_host,

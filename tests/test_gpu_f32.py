@@ -126,3 +126,19 @@ def test_f32_three_stored_terms_equal_the_six_term_problem(shape):
     from gpu_util import gpu_run
     plain = gpu_run(A6, B6, C)
     assert np.array_equal(_gpu(shape, A, B, C).view(np.uint32), plain.view(np.uint32))
+
+
+@pytest.mark.parametrize("shape", [(1, 256, 512, 512), (2, 40, 63, 36), (1, 16, 1024, 1024)])
+def test_f32_matmul_never_reads_c(shape):
+    b, m, k, n = shape
+    A, B, C = _draw(shape, 41 + sum(shape), "int")
+    dA, dB = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
+    dC = torch.full((b, m, n), float("nan"), device="cuda")
+    mb.morello_matmul_f32(b, m, k, n, dA, dB, dC)
+    st, detail = mb.morello_read_device_status()
+    assert st == mb.MORELLO_OK, hex(detail)
+    assert_bit_exact(dC.cpu().numpy(), oracle.matmul_accum_f32(b, m, k, n, A, B, np.zeros_like(C)), "f32 matmul %s" % (shape,))
+    dC.fill_(5.0)
+    mb.morello_matmul_f32(b, m, 0, n, dA, dB, dC)          # an empty sum: C = 0
+    torch.cuda.synchronize()
+    assert float(dC.abs().max()) == 0.0
