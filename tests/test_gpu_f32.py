@@ -104,6 +104,7 @@ def test_f32_empty_and_bad_arguments():
     (1, 8, 4096, 256),       # ... with k slices inside a cluster
     (1, 300, 4096, 264),     # tile kernel with k slices through the workspace
     (1, 64, 64, 128),        # one k block per term
+    (40, 16, 128, 1024),     # 320 (batch, strip) items: the operand-swapped kernel's persistent form
 ])
 def test_f32_three_stored_terms_equal_the_six_term_problem(shape):
     """With k % 64 == 0 the library stores the three bf16 terms of A and B once and lets the
