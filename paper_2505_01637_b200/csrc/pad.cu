@@ -50,10 +50,28 @@ pad_bf16_kernel(const uint16_t* __restrict__ src, uint4* __restrict__ dst, int64
   if (r < rows_in) {
     const uint16_t* row = src + (bb * rows_in + r) * cols_in;
     const int64_t c0 = g * 8;
+    const uint16_t* at = row + c0;
+    if (c0 + 8 <= cols_in) {
+      // Eight elements inside the row: 32-bit loads where the address allows (the source rows
+      // are only 2-byte aligned), 4 or 5 loads instead of 8.
+      if ((reinterpret_cast<uintptr_t>(at) & 2u) == 0) {
+        const uint32_t* q = reinterpret_cast<const uint32_t*>(at);
+        w[0] = q[0]; w[1] = q[1]; w[2] = q[2]; w[3] = q[3];
+      } else {
+        const uint32_t h0 = at[0], h7 = at[7];
+        const uint32_t* q = reinterpret_cast<const uint32_t*>(at + 1);
+        const uint32_t x0 = q[0], x1 = q[1], x2 = q[2];
+        w[0] = h0 | (x0 << 16);
+        w[1] = (x0 >> 16) | (x1 << 16);
+        w[2] = (x1 >> 16) | (x2 << 16);
+        w[3] = (x2 >> 16) | (h7 << 16);
+      }
+    } else {
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const uint32_t v = (c0 + e < cols_in) ? (uint32_t)row[c0 + e] : 0u;
-      w[e >> 1] |= v << ((e & 1) * 16);
+      for (int e = 0; e < 8; ++e) {
+        const uint32_t v = (c0 + e < cols_in) ? (uint32_t)at[e] : 0u;
+        w[e >> 1] |= v << ((e & 1) * 16);
+      }
     }
   }
   dst[idx] = make_uint4(w[0], w[1], w[2], w[3]);
