@@ -8,21 +8,34 @@ One JSON line on stdout.  A step is one MatmulAccum call on the headline
 workload, the 1 x 2048 x 16384 vector-matrix multiply: `value` is its
 algorithmic bytes (A and B read once, C read and written once) per second with
 all operands resident in HBM; the B matrix rotates over 8 distinct 64 MiB
-buffers so that no call finds its input in L2.  `e2e` is the same metric
-through the host-buffer entry point, host<->device copies inside the timed
-region.  `configs` reports the other shapes (GEMM ones in TFLOP/s), each
-against its own roofline.  With --gpus N every rank runs an independent replica
-(the operation has no exchange step); the time is the maximum over ranks.
+buffers so that no call finds its input in L2.
+
+How the headline is timed: every rotating buffer set is called once (untimed,
+so that no first-use cost of a buffer lands in the timed region), then W
+warm-up steps, then the K-step loop runs R times back to back on the stream
+(R >= 25 and at least 50 ms of work), each loop bracketed by its own pair of
+CUDA events, the whole region by a barrier + synchronize on both sides.
+`ms_per_step` is the MEDIAN loop divided by K; the minimum, maximum and mean
+are printed beside it, and `clocks` describes exactly that region.
+
+`e2e` is the same metric through the host-buffer entry point, host<->device
+copies inside the timed region.  `configs` reports the other shapes (GEMM ones
+in TFLOP/s), each against its own roofline, and `cpu_baselines` the CPU oracle
+timed on this machine's host cores for every config (a baseline, not the
+target).  With --gpus N every rank runs an independent replica (the operation
+has no exchange step); the time is the maximum over ranks.  Started without a
+torchrun environment, --gpus N > 1 launches the N ranks itself.
 
 --impl reference times the CPU oracle (the only baseline there is: the paper
-ships no code) on this machine's host cores, on a bounded sample of the same
-workload."""
+ships no code) on this machine's host cores, on the same workload."""
 from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
+import subprocess
 import sys
 import threading
 import time
@@ -38,9 +51,19 @@ from paper_2505_01637_b200 import workloads as w
 METRIC = "bf16->f32 MatmulAccum: GEMV HBM GB/s & GEMM TFLOP/s, % of B200 roofline"
 NOMINAL_HBM_GBS = 8000.0
 NOMINAL_BF16_TFLOPS = 2250.0
+TARGET_HBM_FRAC_OF_NOMINAL = 0.80       # the vector-matrix multiply: >= 80 % of HBM bandwidth
+TARGET_TENSOR_FRAC_OF_NOMINAL = 0.70    # the large GEMMs: >= 70 % of the dense bf16 peak
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 HEADLINE = 1            # index into workloads.CONFIGS: the 1 x 2048 x 16384 GEMV
 ROTATE = 8              # distinct B buffers: 8 x 64 MiB = 512 MiB > 4 x the 126 MB L2
+MIN_LOOPS = 25          # the K-step loop is repeated at least this often ...
+MIN_TIMED_SECONDS = 0.05    # ... and until this much work has been timed
+MAX_LOOPS = 4000
+
+
+def workload_name(cfg):
+    """The string both arms print as config.workload."""
+    return "%s b,m,k,n=%s bf16 x bf16 -> f32 accumulate" % (cfg.name, list(cfg.shape))
 
 
 def load_peaks():
@@ -114,7 +137,7 @@ class ClockSampler:
                 self.samples.append((time.perf_counter(), mhz, reasons, power))
             except Exception:
                 pass
-            time.sleep(0.002)
+            time.sleep(0.001)
 
     def start(self):
         if self._h is not None:
@@ -127,13 +150,12 @@ class ClockSampler:
             self._thread.join(timeout=2)
 
     def summary(self, windows):
-        """Median clock and the reasons seen inside the (t0, t1) windows."""
+        """Median clock and the reasons seen inside the (t0, t1) windows only."""
         names = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
                  0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
                  0x2: "applications_clocks_setting", 0x10: "sync_boost",
                  0x100: "display_clock_setting"}
-        inside = [s for s in self.samples if any(t0 <= s[0] <= t1 for (t0, t1) in windows)]
-        use = inside or self.samples
+        use = [s for s in self.samples if any(t0 <= s[0] <= t1 for (t0, t1) in windows)]
         if not use:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
         mask = 0
@@ -141,9 +163,9 @@ class ClockSampler:
             mask |= s[2]
         powers = [s[3] for s in use if s[3] is not None]
         return {"sm_mhz": statistics.median(s[1] for s in use), "sm_max_mhz": self.max_mhz,
+                "sm_mhz_min": min(s[1] for s in use),
                 "reasons": sorted(names[b] for b in names if mask & b),
-                "samples": len(use), "samples_in_timed_regions": len(inside),
-                "power_w_max": max(powers) if powers else None}
+                "samples": len(use), "power_w_max": max(powers) if powers else None}
 
 
 def nvml_index(local: int) -> int:
@@ -155,37 +177,64 @@ def nvml_index(local: int) -> int:
     return local
 
 
-# ---------------------------------------------------------------- reference arm
-def oracle_sample(cfg_index, budget_s=8.0, threads=None):
-    """Times the CPU oracle, as it stands, on a bounded sample of a config.
-    Returns (seconds, macs, description, threads)."""
+# ------------------------------------------------------- the CPU oracle, timed
+def cfg5_row_sample(cfg):
+    """The seeded row sample a config too large to run whole is timed on: the first and last
+    128 rows of batch 0 plus 32 seeded random rows of every batch (all columns)."""
+    b, m, _, _ = cfg.shape
+    rng = np.random.Generator(np.random.Philox(77))
+    rows = set(range(min(128, m))) | set(range(max(0, m - 128), m))
+    for beta in range(b):
+        rows |= {beta * m + int(i) for i in rng.choice(m, size=min(32, m), replace=False)}
+    return np.array(sorted(rows), dtype=np.int64)
+
+
+def oracle_time(cfg_index, threads=None, budget_s=3.0, host=None):
+    """Times the CPU oracle, as it stands, on one config: the whole problem (repeated for
+    about budget_s when it is short), or, beyond 2e11 multiply-adds, a seeded row sample whose
+    time is extrapolated to the whole problem and labelled so.  Returns a dict."""
     import oracle
-    if threads:
-        oracle.set_num_threads(threads)
-    cfg = w.CONFIGS[cfg_index]
-    b, m, k, n = cfg.shape
-    if cfg.macs <= 2e9:                       # whole problem per repetition
-        A, B, C = w.make_config(cfg_index)
-        oracle.matmul_accum(b, m, k, n, A, B, C)                     # page in, spin up threads
-        reps, t0 = 0, time.perf_counter()
-        while True:
-            oracle.matmul_accum(b, m, k, n, A, B, C)
-            reps += 1
+    all_threads = oracle.num_threads()
+    oracle.set_num_threads(threads or all_threads)
+    try:
+        cfg = w.CONFIGS[cfg_index]
+        b, m, k, n = cfg.shape
+        A, B, C = host if host is not None else w.make_config(cfg_index)
+        used = oracle.num_threads()
+        if cfg.macs <= 2e11:
+            if cfg.macs <= 2e9:
+                oracle.matmul_accum(b, m, k, n, A, B, C)          # page in, spin the threads up
+            reps, t0 = 0, time.perf_counter()
+            while True:
+                oracle.matmul_accum(b, m, k, n, A, B, C)
+                reps += 1
+                el = time.perf_counter() - t0
+                if el >= budget_s or reps >= 2000:
+                    break
+            sec = el / reps
+            what = "whole problem, mean of %d repetition%s" % (reps, "" if reps == 1 else "s")
+            extrapolated = False
+        else:
+            rows = cfg5_row_sample(cfg)
+            t0 = time.perf_counter()
+            oracle.matmul_accum_rows(b, m, k, n, A, B, C, rows, want_abs=False)
             el = time.perf_counter() - t0
-            if el >= budget_s or reps >= 2000:
-                break
-        return el / reps, cfg.macs, "whole problem, mean of %d repetitions" % reps, oracle.num_threads()
-    # a row sample of one batch of a large problem
-    A, B, C = w.make(1, m, k, n, 1000 * cfg_index, cfg.ab, cfg.c)
-    nrows = max(oracle.num_threads(), int(8e9 // (k * n)))
-    rows = np.linspace(0, m - 1, num=min(nrows, m)).astype(np.int64)
-    t0 = time.perf_counter()
-    oracle.matmul_accum_rows(1, m, k, n, A, B, C, rows, want_abs=False)
-    el = time.perf_counter() - t0
-    return el, len(rows) * k * n, "%d of %d rows of batch 0, all columns" % (len(rows), b * m), oracle.num_threads()
+            sec = el * (b * m) / len(rows)
+            what = ("sampled: %d of %d rows (first and last 128 of batch 0, 32 seeded rows per batch), "
+                    "all columns, %.2f s; whole-config time extrapolated" % (len(rows), b * m, el))
+            extrapolated = True
+        return {"name": cfg.name, "shape": list(cfg.shape), "cores": used, "seconds": sec,
+                "GMACps": cfg.macs / sec / 1e9, "GBps": cfg.algorithmic_bytes / sec / 1e9,
+                "TFLOPs": cfg.flops / sec / 1e12, "sample": what, "extrapolated": extrapolated,
+                "kind": "oracle", "label": "baseline, not the target"}
+    finally:
+        oracle.set_num_threads(all_threads)
 
 
 def run_reference(args):
+    """The reference arm: the oracle on the host cores, on the headline workload.  A step is
+    the whole vector-matrix multiply; the K-step loop is repeated like the GPU arm's and the
+    median loop is reported."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
@@ -194,24 +243,28 @@ def run_reference(args):
     oracle.build()
     b, m, k, n = cfg.shape
     A, B, C = w.make_config(HEADLINE)
-    for _ in range(max(args.warmup, 1)):
-        oracle.matmul_accum(b, m, k, n, A, B, C)
     steps = max(1, min(args.steps, 200))
-    t0 = time.perf_counter()
-    for _ in range(steps):
+    for _ in range(max(args.warmup, 3)):
         oracle.matmul_accum(b, m, k, n, A, B, C)
-    el = time.perf_counter() - t0
+    loops, t_begin = [], time.perf_counter()
+    while len(loops) < 5 or (time.perf_counter() - t_begin < 3.0 and len(loops) < 200):
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            oracle.matmul_accum(b, m, k, n, A, B, C)
+        loops.append(time.perf_counter() - t0)
+    el = statistics.median(loops)
     gbs = cfg.algorithmic_bytes * steps / el / 1e9
+    sample = "whole problem per step, median of %d loops of %d steps" % (len(loops), steps)
     line = {
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s",
-        "n_gpus": args.gpus, "steps": steps, "warmup": max(args.warmup, 1),
+        "n_gpus": args.gpus, "steps": steps, "warmup": max(args.warmup, 3),
         "ms_per_step": el / steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "%s b,m,k,n=%s" % (cfg.name, list(cfg.shape)),
+        "config": {"workload": workload_name(cfg),
                    "note": "CPU oracle (double accumulation) on the host cores; each step is "
                            "the whole vector-matrix multiply"},
         "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": oracle.num_threads(),
-                         "kind": "oracle", "sample": "whole problem per step, %d steps" % steps},
+                         "kind": "oracle", "sample": sample},
         "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -236,69 +289,118 @@ def whole_job_value(units_per_rank_per_step, steps, world, seconds):
     return world * units_per_rank_per_step * steps / seconds
 
 
+def loop_count(pilot_seconds):
+    """How often the K-step loop is repeated, from the time of one pilot loop."""
+    if pilot_seconds <= 0:
+        return MIN_LOOPS
+    return int(min(MAX_LOOPS, max(MIN_LOOPS, math.ceil(MIN_TIMED_SECONDS / pilot_seconds))))
+
+
+def spread(loops, steps):
+    """Per-step statistics (microseconds) of a list of K-step loop times (seconds)."""
+    us = [x / steps * 1e6 for x in loops]
+    return {"loops": len(us), "us_per_step_median": statistics.median(us), "us_per_step_min": min(us),
+            "us_per_step_max": max(us), "us_per_step_mean": sum(us) / len(us),
+            "us_per_step_p10": sorted(us)[len(us) // 10], "us_per_step_p90": sorted(us)[(9 * len(us)) // 10]}
+
+
+def timed_loops(torch, fn, steps, loops, first_step=0):
+    """Enqueues `loops` back-to-back loops of `steps` calls of fn(i), an event between
+    consecutive loops; returns the loops' times in seconds.  The caller synchronises before."""
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(loops + 1)]
+    i = first_step
+    ev[0].record()
+    for r in range(loops):
+        for _ in range(steps):
+            fn(i)
+            i += 1
+        ev[r + 1].record()
+    torch.cuda.synchronize()
+    return [ev[r].elapsed_time(ev[r + 1]) * 1e-3 for r in range(loops)]
+
+
 def time_calls(torch, fn, steps, warmup):
     """fn(i) enqueues step i on the current stream; returns seconds for `steps` steps."""
     for i in range(warmup):
         fn(i)
     torch.cuda.synchronize()
-    start = torch.cuda.Event(enable_timing=True)
-    stop = torch.cuda.Event(enable_timing=True)
-    start.record()
-    for i in range(steps):
-        fn(i)
-    stop.record()
-    torch.cuda.synchronize()
-    return start.elapsed_time(stop) * 1e-3
+    return timed_loops(torch, fn, steps, 1)[0]
 
 
-def bench_config(torch, mb, idx, iters, warmup, peaks, windows, path=None, split_k=0, op="matmul_accum"):
-    """Device-timed throughput of one config (inputs resident, rotating when small)."""
+def rotating_sets(in_bytes):
+    return max(1, min(ROTATE, int(np.ceil(512 * 2 ** 20 / in_bytes))))
+
+
+def bench_calls(torch, mb, name, op, shape, dev_sets, call_one, iters, warmup, peaks, windows, alg_bytes,
+                path_name, extra=None):
+    """Device-timed throughput of one arm: `dev_sets` are its rotating operand sets (already on
+    the device), call_one(set) enqueues one call.  Best of three timed loops, the mean beside it."""
+    b, m, k, n = shape
+    sets = len(dev_sets)
+
+    def step(i):
+        rc = call_one(dev_sets[i % sets])
+        if rc != 0:
+            raise mb.MorelloError(rc, "bench %s" % name)
+
+    l0 = mb.morello_launch_count()
+    for s in range(sets):                      # every set once: first-use costs stay untimed
+        step(s)
+    per_call = (mb.morello_launch_count() - l0) // sets
+    t0 = time.perf_counter()
+    loops = [time_calls(torch, step, iters, warmup if r == 0 else 3) for r in range(3)]
+    windows.append((t0, time.perf_counter()))
+    st, detail = mb.morello_read_device_status()
+    if st != 0:
+        raise RuntimeError("device status %d (0x%x) after %s" % (st, detail, name))
+    sec = min(loops) / iters
+    flops = 2.0 * b * m * k * n
+    gbs, tfl = alg_bytes / sec / 1e9, flops / sec / 1e12
+    rec = {"name": name, "op": op, "shape": list(shape), "path": path_name, "us_per_call": sec * 1e6,
+           "us_per_call_mean_of_3_loops": sum(loops) / len(loops) / iters * 1e6,
+           "GBps": gbs, "TFLOPs": tfl, "iters": iters, "launches_per_call": int(per_call),
+           "rotating_sets": sets,
+           "frac_hbm_measured": gbs / peaks["hbm_gbs"], "frac_hbm_nominal": gbs / NOMINAL_HBM_GBS,
+           "frac_tensor_measured_burst": tfl / peaks["bf16_tflops"],
+           "frac_tensor_nominal": tfl / NOMINAL_BF16_TFLOPS}
+    if extra:
+        rec.update(extra)
+    return rec
+
+
+def to_device(torch, A, B, C):
+    return (torch.from_numpy(A.view(np.int16)).cuda(), torch.from_numpy(B.view(np.int16)).cuda(),
+            torch.from_numpy(np.ascontiguousarray(C)).cuda())
+
+
+def bench_config(torch, mb, idx, iters, warmup, peaks, windows, path=None, split_k=0, op="matmul_accum",
+                 host=None):
+    """One named config (inputs resident, rotating when small) through the forced entry point
+    (path None = the selector's choice)."""
     cfg = w.CONFIGS[idx]
     b, m, k, n = cfg.shape
     in_bytes = 2 * b * m * k + 2 * b * k * n + 4 * b * m * n
-    sets = max(1, min(ROTATE, int(np.ceil(512 * 2 ** 20 / in_bytes))))
-    A, B, C = w.make_config(idx)
+    sets = rotating_sets(in_bytes)
+    A, B, C = host if host is not None else w.make_config(idx)
     dev = []
     for s in range(sets):
         if s == 0:
             As, Bs = A, B
         else:                                   # fresh values for every rotating copy
             As, Bs, _ = w.make(b, m, k, n, 1000 * idx + 100 * s, cfg.ab, "zeros")
-        dev.append((torch.from_numpy(As.view(np.int16)).cuda(), torch.from_numpy(Bs.view(np.int16)).cuda(),
-                    torch.from_numpy(C.copy()).cuda()))
-    ptrs = [(a.data_ptr(), bb.data_ptr(), c.data_ptr()) for (a, bb, c) in dev]
+        dev.append(to_device(torch, As, Bs, C.copy()))
     stream = torch.cuda.current_stream().cuda_stream
     call = mb.lib().morello_matmul_accum_forced if op == "matmul_accum" else mb.lib().morello_matmul_forced
     forced = mb.MORELLO_PATH_AUTO if path is None else path
 
-    def step(i):
-        pa, pb, pc = ptrs[i % sets]
-        rc = call(forced, split_k, b, m, k, n, pa, pb, pc, None, 0, stream)
-        if rc != 0:
-            raise mb.MorelloError(rc, "bench %s" % cfg.name)
+    def call_one(t):
+        return call(forced, split_k, b, m, k, n, t[0].data_ptr(), t[1].data_ptr(), t[2].data_ptr(), None, 0, stream)
 
-    l0 = mb.morello_launch_count()
-    step(0)
-    per_call = mb.morello_launch_count() - l0
-    t0 = time.perf_counter()
-    loops = [time_calls(torch, step, iters, warmup if r == 0 else 3) for r in range(3)]
-    windows.append((t0, time.perf_counter()))
-    sec = min(loops)                          # best of three timed loops; the mean is kept beside it
-    st, detail = mb.morello_read_device_status()
-    if st != 0:
-        raise RuntimeError("device status %d (0x%x) after %s" % (st, detail, cfg.name))
-    us = sec / iters * 1e6
-    alg_bytes = cfg.algorithmic_bytes - (4 * b * m * n if op == "matmul" else 0)   # Matmul never reads C
-    gbs = alg_bytes / (sec / iters) / 1e9
-    tfl = cfg.flops / (sec / iters) / 1e12
     chosen = mb.morello_select_path(b, m, k, n) if path is None else path
-    rec = {"name": cfg.name, "op": op, "shape": list(cfg.shape), "path": "tcgen05" if chosen == 1 else "skinny",
-           "us_per_call": us, "us_per_call_mean_of_3_loops": sum(loops) / len(loops) / iters * 1e6, "GBps": gbs, "TFLOPs": tfl, "iters": iters, "launches_per_call": per_call,
-           "rotating_sets": sets,
-           "frac_hbm_measured": gbs / peaks["hbm_gbs"], "frac_hbm_nominal": gbs / NOMINAL_HBM_GBS,
-           "frac_tensor_measured_burst": tfl / peaks["bf16_tflops"],
-           "frac_tensor_measured_sustained": tfl / peaks["bf16_tflops_sustained"],
-           "frac_tensor_nominal": tfl / NOMINAL_BF16_TFLOPS}
+    alg = cfg.algorithmic_bytes - (4 * b * m * n if op == "matmul" else 0)   # Matmul never reads C
+    rec = bench_calls(torch, mb, cfg.name, op, cfg.shape, dev, call_one, iters, warmup, peaks, windows, alg,
+                      "tcgen05" if chosen == 1 else "skinny",
+                      {"route": mb.morello_describe_route(b, m, k, n)} if path is None else None)
     del dev
     torch.cuda.empty_cache()
     return rec
@@ -306,44 +408,26 @@ def bench_config(torch, mb, idx, iters, warmup, peaks, windows, path=None, split
 
 def bench_shape(torch, mb, name, shape, iters, peaks, windows, note):
     """A shape outside the named configs, through the plain entry point: the selector's other
-    routes (k slices through the workspace, padded copies, the flat FMA form, the single row
-    on the tensor kernel).  Inputs rotate like bench_config's; normal(0, 1/sqrt(k)) values."""
+    routes and the mid-sized shapes.  Inputs rotate like bench_config's; normal(0, 1/sqrt(k))."""
     b, m, k, n = shape
     in_bytes = 2 * b * m * k + 2 * b * k * n + 4 * b * m * n
-    sets = max(1, min(ROTATE, int(np.ceil(512 * 2 ** 20 / in_bytes))))
     dev = []
-    for s_ in range(sets):
+    for s_ in range(rotating_sets(in_bytes)):
         As, Bs, Cs = w.make(b, m, k, n, 9000 + 10 * s_ + (m + k + n) % 7, "normal_rsqrtk", "zeros")
-        dev.append((torch.from_numpy(As.view(np.int16)).cuda(), torch.from_numpy(Bs.view(np.int16)).cuda(),
-                    torch.from_numpy(Cs).cuda()))
-    ptrs = [(a.data_ptr(), bb.data_ptr(), c.data_ptr()) for (a, bb, c) in dev]
+        dev.append(to_device(torch, As, Bs, Cs))
     stream = torch.cuda.current_stream().cuda_stream
     call = mb.lib().morello_matmul_accum
 
-    def step(i):
-        pa, pb, pc = ptrs[i % sets]
-        rc = call(b, m, k, n, pa, pb, pc, stream)
-        if rc != 0:
-            raise mb.MorelloError(rc, "bench %s" % name)
+    def call_one(t):
+        return call(b, m, k, n, t[0].data_ptr(), t[1].data_ptr(), t[2].data_ptr(), stream)
 
-    l0 = mb.morello_launch_count()
-    step(0)
-    per_call = mb.morello_launch_count() - l0
-    t0 = time.perf_counter()
-    loops = [time_calls(torch, step, iters, 5 if r == 0 else 3) for r in range(3)]
-    windows.append((t0, time.perf_counter()))
-    sec = min(loops) / iters
-    st, detail = mb.morello_read_device_status()
-    if st != 0:
-        raise RuntimeError("device status %d (0x%x) after %s" % (st, detail, name))
-    alg = in_bytes + 4 * b * m * n
-    flops = 2.0 * b * m * k * n
-    return {"name": name, "op": "matmul_accum", "shape": list(shape),
-            "path": "tcgen05" if mb.morello_select_path(b, m, k, n) == 1 else "skinny",
-            "us_per_call": sec * 1e6, "GBps": alg / sec / 1e9, "TFLOPs": flops / sec / 1e12,
-            "iters": iters, "launches_per_call": per_call, "rotating_sets": sets,
-            "frac_hbm_measured": alg / sec / 1e9 / peaks["hbm_gbs"],
-            "frac_tensor_measured_burst": flops / sec / 1e12 / peaks["bf16_tflops"], "note": note}
+    rec = bench_calls(torch, mb, name, "matmul_accum", shape, dev, call_one, iters, 5, peaks, windows,
+                      in_bytes + 4 * b * m * n,
+                      "tcgen05" if mb.morello_select_path(b, m, k, n) == 1 else "skinny",
+                      {"note": note, "route": mb.morello_describe_route(b, m, k, n)})
+    del dev
+    torch.cuda.empty_cache()
+    return rec
 
 
 def bench_f32_square(torch, mb, peaks, windows, size=2048, iters=20):
@@ -376,86 +460,42 @@ def bench_f32_square(torch, mb, peaks, windows, size=2048, iters=20):
             "bf16_TFLOPs_executed": 6 * flops / sec / 1e12,
             "frac_tensor_measured_burst_of_executed": 6 * flops / sec / 1e12 / peaks["bf16_tflops"],
             "fp32_alu_peak_TFLOPs_for_context": 148 * 128 * 2 * 1.965e9 / 1e12,
-            "iters": iters, "launches_per_call": per_call,
+            "iters": iters, "launches_per_call": int(per_call),
             "note": "inputs split exactly into three bf16 terms; six of nine cross products kept"}
 
 
-def bench_colmajor(torch, mb, idx, iters, peaks, windows):
-    """A config with its B stored column-major (Bt[b][n][k]) through
-    morello_matmul_accum_colmajor_b; inputs rotate like bench_config's."""
+def bench_layout(torch, mb, idx, iters, peaks, windows, strip=0):
+    """A config with its B stored column-major (Bt[b][n][k], strip 0) or packed in strips of
+    `strip` columns (Bp[b][n/strip][k][strip]); inputs rotate like bench_config's."""
     cfg = w.CONFIGS[idx]
     b, m, k, n = cfg.shape
     in_bytes = 2 * b * m * k + 2 * b * k * n + 4 * b * m * n
-    sets = max(1, min(ROTATE, int(np.ceil(512 * 2 ** 20 / in_bytes))))
     dev = []
-    for s_ in range(sets):
-        As, Bs, Cs = w.make(b, m, k, n, 1000 * idx + 100 * s_ + 50, cfg.ab, "zeros")
-        Bt = np.ascontiguousarray(Bs.transpose(0, 2, 1))
-        dev.append((torch.from_numpy(As.view(np.int16)).cuda(), torch.from_numpy(Bt.view(np.int16)).cuda(),
-                    torch.from_numpy(Cs).cuda()))
-    ptrs = [(a.data_ptr(), bb.data_ptr(), c.data_ptr()) for (a, bb, c) in dev]
+    for s_ in range(rotating_sets(in_bytes)):
+        As, Bs, Cs = w.make(b, m, k, n, 1000 * idx + 100 * s_ + (70 if strip else 50), cfg.ab, "zeros")
+        Bl = w.pack_b(Bs, strip) if strip else np.ascontiguousarray(Bs.transpose(0, 2, 1))
+        dev.append(to_device(torch, As, Bl, Cs))
     stream = torch.cuda.current_stream().cuda_stream
-    call = mb.lib().morello_matmul_accum_colmajor_b
+    if strip:
+        call = mb.lib().morello_matmul_accum_packed_b
+        op, first = "matmul_accum_packed_b", strip
+    else:
+        call = mb.lib().morello_matmul_accum_colmajor_b
+        op, first = "matmul_accum_colmajor_b", 0
 
-    def step(i):
-        pa, pb, pc = ptrs[i % sets]
-        rc = call(0, b, m, k, n, pa, pb, pc, stream)
-        if rc != 0:
-            raise mb.MorelloError(rc, "bench col-major %s" % cfg.name)
+    def call_one(t):
+        return call(first, b, m, k, n, t[0].data_ptr(), t[1].data_ptr(), t[2].data_ptr(), stream)
 
-    l0 = mb.morello_launch_count()
-    step(0)
-    per_call = mb.morello_launch_count() - l0
-    t0 = time.perf_counter()
-    loops = [time_calls(torch, step, iters, 5 if r == 0 else 3) for r in range(3)]
-    windows.append((t0, time.perf_counter()))
-    sec = min(loops) / iters
-    return {"name": cfg.name, "op": "matmul_accum_colmajor_b", "shape": list(cfg.shape), "path": "tcgen05",
-            "us_per_call": sec * 1e6, "GBps": cfg.algorithmic_bytes / sec / 1e9, "TFLOPs": cfg.flops / sec / 1e12,
-            "iters": iters, "launches_per_call": per_call, "rotating_sets": sets,
-            "frac_hbm_measured": cfg.algorithmic_bytes / sec / 1e9 / peaks["hbm_gbs"],
-            "frac_tensor_measured_burst": cfg.flops / sec / 1e12 / peaks["bf16_tflops"]}
-
-
-def bench_packed(torch, mb, idx, strip, iters, peaks, windows):
-    """A config with its B packed in strips of `strip` columns (Bp[b][n/strip][k][strip])
-    through morello_matmul_accum_packed_b; inputs rotate like bench_config's."""
-    cfg = w.CONFIGS[idx]
-    b, m, k, n = cfg.shape
-    in_bytes = 2 * b * m * k + 2 * b * k * n + 4 * b * m * n
-    sets = max(1, min(ROTATE, int(np.ceil(512 * 2 ** 20 / in_bytes))))
-    dev = []
-    for s_ in range(sets):
-        As, Bs, Cs = w.make(b, m, k, n, 1000 * idx + 100 * s_ + 70, cfg.ab, "zeros")
-        dev.append((torch.from_numpy(As.view(np.int16)).cuda(),
-                    torch.from_numpy(w.pack_b(Bs, strip).view(np.int16)).cuda(), torch.from_numpy(Cs).cuda()))
-    ptrs = [(a.data_ptr(), bb.data_ptr(), c.data_ptr()) for (a, bb, c) in dev]
-    stream = torch.cuda.current_stream().cuda_stream
-    call = mb.lib().morello_matmul_accum_packed_b
-
-    def step(i):
-        pa, pb, pc = ptrs[i % sets]
-        rc = call(strip, b, m, k, n, pa, pb, pc, stream)
-        if rc != 0:
-            raise mb.MorelloError(rc, "bench packed %s" % cfg.name)
-
-    l0 = mb.morello_launch_count()
-    step(0)
-    per_call = mb.morello_launch_count() - l0
-    t0 = time.perf_counter()
-    loops = [time_calls(torch, step, iters, 5 if r == 0 else 3) for r in range(3)]
-    windows.append((t0, time.perf_counter()))
-    sec = min(loops) / iters
-    return {"name": cfg.name, "op": "matmul_accum_packed_b", "strip": strip, "shape": list(cfg.shape),
-            "path": "tcgen05", "us_per_call": sec * 1e6, "GBps": cfg.algorithmic_bytes / sec / 1e9,
-            "TFLOPs": cfg.flops / sec / 1e12, "iters": iters, "launches_per_call": per_call,
-            "rotating_sets": sets, "frac_hbm_measured": cfg.algorithmic_bytes / sec / 1e9 / peaks["hbm_gbs"],
-            "frac_tensor_measured_burst": cfg.flops / sec / 1e12 / peaks["bf16_tflops"]}
+    rec = bench_calls(torch, mb, cfg.name, op, cfg.shape, dev, call_one, iters, 5, peaks, windows,
+                      cfg.algorithmic_bytes, "tcgen05", {"strip": strip} if strip else None)
+    del dev
+    torch.cuda.empty_cache()
+    return rec
 
 
 def run_case(args):
-    """One configuration alone, device-timed: the command the ncu captures under
-    profiles/ were taken with, and the unit of the sweeps quoted in the design notes."""
+    """One configuration alone, device-timed: the command the ncu captures under profiles/
+    were taken with, and the unit of single-shape sweeps."""
     import torch
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
@@ -470,11 +510,21 @@ def run_case(args):
         print(json.dumps(rec))
         return 0
     rec = bench_config(torch, mb, args.case - 1, args.steps, args.warmup, peaks, [], path=path,
-                       split_k=args.split)
+                       split_k=args.split, op=args.op)
     rec["case"] = args.case
     rec["split_k_knob"] = args.split
     print(json.dumps(rec))
     return 0
+
+
+def tensor_roofline(rec, peaks, peak_kind, traffic):
+    return {"bound": "tensor", "achieved": rec["TFLOPs"], "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+            "frac": rec["TFLOPs"] / peaks["bf16_tflops"], "peak_kind": peak_kind + " (cuBLAS burst)",
+            "frac_of_nominal_2250": rec["TFLOPs"] / NOMINAL_BF16_TFLOPS,
+            "target": "%.0f %% of the nominal 2,250 TFLOP/s" % (100 * TARGET_TENSOR_FRAC_OF_NOMINAL),
+            "target_met": rec["TFLOPs"] / NOMINAL_BF16_TFLOPS >= TARGET_TENSOR_FRAC_OF_NOMINAL,
+            "workload": rec["name"], "us_per_call": rec["us_per_call"], "traffic": traffic.get(rec["name"]),
+            "kernel": rec.get("route", "gemm_kernel")}
 
 
 def run_ours(args):
@@ -516,33 +566,34 @@ def run_ours(args):
             raise mb.MorelloError(rc, "bench step")
 
     sampler.start()
-    # ---- headline: K steps, device-timed, barrier + synchronize on both sides
+    # ---- headline.  Every rotating set once (untimed): tensor maps encoded, pages mapped.
+    for i in range(ROTATE):
+        step(i)
+    torch.cuda.synchronize()
     for i in range(args.warmup):
         step(i)
+    pilot = max_over_ranks(time_calls(torch, step, args.steps, 0), dist, "cuda")   # one more untimed loop
+    loops_n = loop_count(pilot)
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
         torch.cuda.synchronize()
     l0 = mb.morello_launch_count()
-    start = torch.cuda.Event(enable_timing=True)
-    stop = torch.cuda.Event(enable_timing=True)
     t0 = time.perf_counter()
-    start.record()
-    for i in range(args.steps):
-        step(i)
-    stop.record()
-    torch.cuda.synchronize()
-    windows.append((t0, time.perf_counter()))
+    loops = timed_loops(torch, step, args.steps, loops_n)     # ends with a synchronize
+    headline_window = [(t0, time.perf_counter())]
     if dist is not None:
         dist.barrier()
         torch.cuda.synchronize()
     launches = mb.morello_launch_count() - l0
-    sec = start.elapsed_time(stop) * 1e-3
-    sec = max_over_ranks(sec, dist, "cuda")
+    sec = max_over_ranks(statistics.median(loops), dist, "cuda")      # the median K-step loop
     st, detail = mb.morello_read_device_status()
     if st != 0:
         raise RuntimeError("device status %d (0x%x)" % (st, detail))
     value = whole_job_value(cfg.algorithmic_bytes, args.steps, world, sec) / 1e9
+    timing = spread(loops, args.steps)
+    timing["loop_us"] = [round(x * 1e6, 2) for x in loops]
+    timing["whole_region_us_per_step"] = sum(loops) / (len(loops) * args.steps) * 1e6
 
     # ---- the same calls on ONE set of buffers (how the config is worded: "timed warm over 1000
     # calls"); B's 64 MiB fit the 126 MB L2, so this figure is L2-assisted and is not the headline
@@ -551,7 +602,7 @@ def run_ours(args):
         if rc != 0:
             raise mb.MorelloError(rc, "bench step")
     t0 = time.perf_counter()
-    same_us = time_calls(torch, step_same, args.steps, args.warmup) / args.steps * 1e6
+    same_us = time_calls(torch, step_same, max(args.steps, 200), args.warmup) / max(args.steps, 200) * 1e6
     windows.append((t0, time.perf_counter()))
 
     # ---- the same loop replayed from a CUDA graph (launch overhead taken out)
@@ -565,7 +616,7 @@ def run_ours(args):
                 for i in range(ROTATE):
                     rc = call(b, m, k, n, pa, pbs[i], pcs[i], cap)
                     assert rc == 0, rc
-            reps = max(1, args.steps // ROTATE)
+            reps = max(25, args.steps // ROTATE)
             for _ in range(3):
                 g.replay()
             side.synchronize()
@@ -603,89 +654,132 @@ def run_ours(args):
     e2e_value = world * cfg.algorithmic_bytes * e2e_steps / e2e_sec / 1e9
     h2d = 2 * b * m * k + 2 * b * k * n + 4 * b * m * n
     d2h = 4 * b * m * n
+    del hA, hB, hC
 
-    # ---- the other configurations (rank 0 of a single-GPU run only)
-    extra = []
+    # ---- the other configurations (a single-GPU run only)
+    extra, cpu_all = [], []
+    want_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
     if world == 1 and args.configs:
         plan = {0: (1000, 50), 2: (300, 20), 3: (30, 5), 4: (6, 2)}
         for idx in args.configs:
             if idx == HEADLINE or idx not in plan:
                 continue
             iters, wu = plan[idx]
-            extra.append(bench_config(torch, mb, idx, iters, wu, peaks, windows))
+            host = w.make_config(idx)
+            extra.append(bench_config(torch, mb, idx, iters, wu, peaks, windows, host=host))
             if idx == 4:                        # the large config also without the read of C (Matmul)
-                extra.append(bench_config(torch, mb, idx, iters, wu, peaks, windows, op="matmul"))
+                extra.append(bench_config(torch, mb, idx, iters, wu, peaks, windows, op="matmul", host=host))
             if idx == 2:                        # crossover config: also on the path not chosen
                 other = (mb.MORELLO_PATH_TCGEN05
                          if mb.morello_select_path(*w.CONFIGS[2].shape) == mb.MORELLO_PATH_SKINNY
                          else mb.MORELLO_PATH_SKINNY)
                 try:
-                    extra.append(bench_config(torch, mb, idx, 100, wu, peaks, windows, path=other))
+                    extra.append(bench_config(torch, mb, idx, 100, wu, peaks, windows, path=other, host=host))
                 except mb.MorelloError:
                     pass
+            if want_cpu:                        # the oracle on the same inputs, all host cores
+                cpu_all.append(oracle_time(idx, host=host))
+                if idx in (0, 2):
+                    cpu_all.append(oracle_time(idx, threads=1, host=host))
+            del host
     if world == 1 and args.configs:
         extra.append(bench_f32_square(torch, mb, peaks, windows))
-        extra.append(bench_colmajor(torch, mb, HEADLINE, 300, peaks, windows))
+        extra.append(bench_layout(torch, mb, HEADLINE, 300, peaks, windows))
         if 3 in args.configs:
-            extra.append(bench_colmajor(torch, mb, 3, 30, peaks, windows))
+            extra.append(bench_layout(torch, mb, 3, 30, peaks, windows))
         if 2 in args.configs:
-            extra.append(bench_packed(torch, mb, 2, 64, 300, peaks, windows))
+            extra.append(bench_layout(torch, mb, 2, 300, peaks, windows, strip=64))
         for name, shape, iters, note in (
                 ("route_gemv_long_k", (1, 1, 8192, 16384), 100, "single row on the operand-swapped tensor kernel"),
                 ("route_k_slices", (1, 512, 16384, 2048), 100, "few tiles, long k: k slices through the workspace + reduce launch"),
-                ("route_padded_copies", (1, 2048, 2047, 2049), 50, "k, n not multiples of 8: zero-padded copies, tensor kernels, unpad-add"),
-                ("route_flat_gemv", (1, 1, 2048, 16383), 100, "n odd, one row: FMA kernel reading aligned 16-byte granules")):
+                ("route_padded_copies", (1, 2048, 2047, 2049), 50, "k, n not multiples of 8: zero-padded copies, tensor kernels"),
+                ("route_flat_gemv", (1, 1, 2048, 16383), 100, "n odd, one row: FMA kernel reading aligned 16-byte granules"),
+                ("mid_128x2048x16384", (1, 128, 2048, 16384), 200, "128 rows on a streaming shape"),
+                ("mid_256x4096x4096", (1, 256, 4096, 4096), 200, "few tiles, k slices"),
+                ("mid_512x4096x4096", (1, 512, 4096, 4096), 200, "few tiles"),
+                ("mid_256x8192x8192", (1, 256, 8192, 8192), 100, "one row of pair tiles, long k")):
             extra.append(bench_shape(torch, mb, name, shape, iters, peaks, windows, note))
     sampler.stop()
-    clocks = sampler.summary(windows)
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        sec_cpu, macs, what, threads = oracle_sample(HEADLINE)
-        cpu = {"value": cfg.algorithmic_bytes * (macs / cfg.macs) / sec_cpu / 1e9, "unit": "GB/s",
-               "cores": threads, "kind": "oracle", "sample": what, "seconds_per_step": sec_cpu}
+    if want_cpu:
+        head = oracle_time(HEADLINE, budget_s=6.0, host=(A, B0, C))
+        cpu = {"value": head["GBps"], "unit": "GB/s", "cores": head["cores"], "kind": "oracle",
+               "sample": head["sample"], "seconds_per_step": head["seconds"]}
+        cpu_all.insert(0, head)
+        cpu_all.insert(1, oracle_time(HEADLINE, threads=1, host=(A, B0, C)))
+        by_name = {}
+        for r in extra:                         # GPU time / oracle time on the same config
+            if r["op"] == "matmul_accum" and r.get("route") is not None:
+                by_name.setdefault(r["name"], r["us_per_call"] * 1e-6)
+        by_name[cfg.name] = sec / args.steps
+        for c in cpu_all:
+            if c["name"] in by_name:
+                c["gpu_over_oracle_speed"] = c["seconds"] / by_name[c["name"]]
 
     if rank == 0:
         per_launch_gbs = cfg.algorithmic_bytes * args.steps / (sec * 1e9)
         line = {
-            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": sec / args.steps * 1e3, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": "%s b,m,k,n=%s bf16 x bf16 -> f32 accumulate" % (cfg.name, list(cfg.shape)),
-                       "l2": "B rotates over %d distinct 64 MiB buffers (512 MiB > 4 x L2), no flush needed" % ROTATE,
-                       "inputs": "A,B uniform[-1,1) bf16, C zeros; Philox seeds 1000*cfg+batch",
-                       "parallelism": "replicas only (no exchange step)" if world > 1 else "1 GPU",
-                       "launch": "back-to-back C-ABI calls on one stream"},
-            "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-            "gpu_launches": int(launches),
-            "roofline": {"bound": "hbm", "achieved": per_launch_gbs, "peak": peaks["hbm_gbs"],
-                         "unit": "GB/s", "frac": per_launch_gbs / peaks["hbm_gbs"],
-                         "peak_kind": peak_kind, "frac_of_nominal_8TBs": per_launch_gbs / NOMINAL_HBM_GBS,
-                         "traffic": traffic.get(cfg.name), "kernel": "gemv_stream_kernel<1>"},
+            "configs": extra,
+            "cpu_baselines": cpu_all,
+            "cpu_baselines_note": "the CPU oracle as it stands on this machine's host cores: a baseline, not the target",
+            "inputs_crc32": {"A": w.crc32(A), "B0": w.crc32(B0), "C": w.crc32(C)},
             "graph_replay_us_per_call": graph_us,
             "same_buffer_us_per_call": same_us,
             "same_buffer_note": "one B buffer re-read every call: 64 MiB < L2, L2-assisted, not an HBM figure",
-            "inputs_crc32": {"A": w.crc32(A), "B0": w.crc32(B0), "C": w.crc32(C)},
+            "clocks_other_arms": sampler.summary(windows),
+            "timing": timing,
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec / args.steps * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": workload_name(cfg),
+                       "l2": "B rotates over %d distinct 64 MiB buffers (512 MiB > 4 x L2), no flush needed" % ROTATE,
+                       "inputs": "A,B uniform[-1,1) bf16, C zeros; Philox seeds 1000*cfg+batch",
+                       "parallelism": "replicas only (no exchange step)" if world > 1 else "1 GPU",
+                       "launch": "back-to-back C-ABI calls on one stream",
+                       "pretouch": "each of the %d rotating buffer sets called once before the warm-up (untimed)" % ROTATE,
+                       "timed": "%d back-to-back loops of %d steps, an event between loops; ms_per_step = median loop / steps"
+                                % (len(loops), args.steps)},
+            "clocks": sampler.summary(headline_window),
+            "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+            "gpu_launches": int(launches),
+            "gpu_launches_per_step": launches / float(len(loops) * args.steps),
             "cpu_baseline": cpu,
-            "configs": extra,
+            "roofline": {"bound": "hbm", "achieved": per_launch_gbs, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": per_launch_gbs / peaks["hbm_gbs"],
+                         "peak_kind": peak_kind, "frac_of_nominal_8TBs": per_launch_gbs / NOMINAL_HBM_GBS,
+                         "target": "%.0f %% of the nominal 8,000 GB/s" % (100 * TARGET_HBM_FRAC_OF_NOMINAL),
+                         "target_met": per_launch_gbs / NOMINAL_HBM_GBS >= TARGET_HBM_FRAC_OF_NOMINAL,
+                         "traffic": traffic.get(cfg.name), "kernel": "gemv_stream_kernel<1>"},
         }
-        gemm = [r for r in extra if r["path"] == "tcgen05" and r["op"] == "matmul_accum"
-                and r["name"].startswith(("cfg4", "cfg5"))]
-        if gemm:
-            best = max(gemm, key=lambda r: r["TFLOPs"])
-            line["roofline_gemm"] = {"bound": "tensor", "achieved": best["TFLOPs"], "peak": peaks["bf16_tflops"],
-                                     "unit": "TFLOP/s", "frac": best["TFLOPs"] / peaks["bf16_tflops"],
-                                     "peak_kind": peak_kind + " (cuBLAS burst)", "workload": best["name"],
-                                     "traffic": traffic.get(best["name"]), "kernel": "gemm_tcgen05"}
+        for r in extra:
+            if r["op"] == "matmul_accum" and r.get("route") is not None and r["name"].startswith("cfg4"):
+                line["roofline_gemm"] = tensor_roofline(r, peaks, peak_kind, traffic)
+            if r["op"] == "matmul_accum" and r.get("route") is not None and r["name"].startswith("cfg5"):
+                line["roofline_gemm_cfg5"] = tensor_roofline(r, peaks, peak_kind, traffic)
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
     return 0
 
 
-def main():
+def free_port():
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def rank_command(n, argv):
+    """The command that starts bench.py as n ranks on this node (one per GPU)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+            "--master-addr", "127.0.0.1", "--master-port", str(free_port()),
+            os.path.abspath(__file__)] + list(argv)
+
+
+def main(argv=None):
+    argv = list(sys.argv[1:] if argv is None else argv)
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
@@ -699,12 +793,16 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "skinny", "tcgen05"],
                     help="kernel family for --case")
     ap.add_argument("--split", type=int, default=0, help="forced split / form knob for --case")
+    ap.add_argument("--op", default="matmul_accum", choices=["matmul_accum", "matmul"], help="operation for --case")
     ap.add_argument("--shape", default="",
                     help="b,m,k,n: time this shape alone through the plain entry point (like --case)")
-    args = ap.parse_args()
+    args = ap.parse_args(argv)
     args.warmup = max(args.warmup, 3)
     args.steps = max(args.steps, 1)
     args.configs = [int(x) - 1 for x in args.configs.split(",") if x.strip()]
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.case or args.shape):
+        # Not under torchrun: start the ranks here; rank 0 prints the line.
+        return subprocess.call(rank_command(args.gpus, argv))
     if args.impl == "reference":
         return run_reference(args)
     if args.case or args.shape:

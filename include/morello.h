@@ -68,7 +68,12 @@ enum {
  * untouched (empty sum).  Scratch memory, when the chosen kernel needs any, is
  * a per-device buffer owned by the library that grows on demand (the only
  * allocation this call can make); concurrent calls on different streams that
- * both need scratch must use morello_matmul_accum_ws instead.
+ * both need scratch must use morello_matmul_accum_ws instead.  Growing the buffer
+ * frees and allocates device memory, which a stream capture does not allow: a call
+ * that would have to grow it while `stream` is being captured returns
+ * MORELLO_ERR_WORKSPACE and touches nothing -- size the buffer with an ordinary call
+ * on the same shape first, or capture morello_matmul_accum_ws.  The same holds for
+ * every entry point below that uses the library's own buffers.
  */
 int morello_matmul_accum(int64_t b, int64_t m, int64_t k, int64_t n,
                          const void* A, const void* B, float* C, void* stream);
@@ -176,10 +181,12 @@ int morello_matmul_f32(int64_t b, int64_t m, int64_t k, int64_t n,
 
 /*
  * End-to-end convenience call on HOST buffers (same layouts): copies A, B and
- * C to library-owned device staging (grown on demand), runs the operation,
- * copies C back and synchronises before returning.  Pinned host memory makes
- * the copies asynchronous with respect to each other but the call still
- * returns only when C_host holds the result.
+ * C to library-owned device staging (one buffer per device, grown on demand), runs
+ * the operation, copies C back and synchronises before returning.  Pinned host memory
+ * makes the copies asynchronous with respect to each other but the call still
+ * returns only when C_host holds the result.  Host threads that call it at the same
+ * time take turns inside the library (the staging buffer is shared), so it is safe
+ * but not concurrent.
  */
 int morello_matmul_accum_host(int64_t b, int64_t m, int64_t k, int64_t n,
                               const void* A_host, const void* B_host, float* C_host);
@@ -189,7 +196,7 @@ int morello_matmul_accum_host(int64_t b, int64_t m, int64_t k, int64_t n,
  * not for the method).  Same operation, computed by the FP32-FMA kernel with the k
  * range cut into `split_k` slices (0 = let the library choose); the slices' partial
  * sums go to a fixed device array of MORELLO_NOALLOC_SCRATCH_BYTES that is part of
- * the library image, so neither this call nor anything it uses ever calls cudaMalloc,
+ * the library image, so neither this call nor anything it uses calls cudaMalloc,
  * cudaFree or an allocating library routine.  It is meant for processes that must not
  * allocate at call time: ones that gave all device memory to their own pool at
  * start-up (a late cudaMalloc may fail there, and while it runs it holds up every
@@ -201,7 +208,12 @@ int morello_matmul_accum_host(int64_t b, int64_t m, int64_t k, int64_t n,
  *    (split_k = 1 needs no scratch and always fits);
  *  - the first call on each device resolves the array's device address (with that
  *    device current) and queries two device attributes; make that first call before
- *    starting any stream capture;
+ *    starting any stream capture.  The CUDA runtime may load a kernel's code onto the
+ *    device the first time that kernel is launched (lazy module loading), which is an
+ *    allocation of the runtime's, not of this library: after one warm-up call per kernel
+ *    variant (row count 1, 2, 4, 8 or 16 of the last chunk, load width, aligned or
+ *    shifted-granule form) -- or with CUDA_MODULE_LOADING=EAGER -- no call changes the
+ *    device's free memory;
  *  - all calls on a device share the one array and it keeps whatever the last call
  *    left in it.  Nothing in it has to be zero beforehand (every word that is read was
  *    written by the same call), but two calls that overlap on the GPU -- different
@@ -232,6 +244,16 @@ size_t morello_noalloc_scratch_limit(void);
  * shapes).  (The single-row choice looks at the device's SM count;
  * 148 SMs are assumed when no device is usable). */
 int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n);
+
+/*
+ * Which kernel, tile and k slices morello_matmul_accum would use for this shape with 16-byte-
+ * aligned operands on the current device (148 SMs assumed when no device is usable), as one line
+ * of text for logs: e.g. "tcgen05 gemm_kernel: a CTA pair per 256 x 256 tile, ...".  `text`
+ * (host memory, `text_bytes` long, caller-owned) receives at most text_bytes - 1 characters and
+ * a terminating NUL.  Enqueues nothing.  Returns MORELLO_OK, MORELLO_ERR_NULL_POINTER for a
+ * missing buffer, or MORELLO_ERR_INVALID_SHAPE.
+ */
+int morello_describe_route(int64_t b, int64_t m, int64_t k, int64_t n, char* text, size_t text_bytes);
 
 /*
  * Run on a given path (MORELLO_PATH_AUTO = selector) with a given split of the
@@ -285,6 +307,16 @@ int morello_read_device_status(void* stream, uint32_t* detail);
  * clears it), MORELLO_ERR_CUDA if it did not.  Faults and hangs nothing.
  */
 int morello_selftest_wait_timeout(uint32_t limit_ms, void* stream);
+
+/*
+ * Host-only self-test of the once-per-device bookkeeping (function attributes such as the
+ * shared-memory opt-in belong to each device's copy of a kernel, so they are set once per
+ * device, not once per process): simulates `calls_per_device` rounds of calls over `devices`
+ * device indices, the first set-up attempt on device 1 failing, and returns how often the
+ * set-up ran -- `devices` + 1 when devices >= 2 and calls_per_device >= 2 (a failure is
+ * retried, a success is remembered).  Needs no GPU; -1 for negative arguments.
+ */
+int morello_selftest_per_device_once(int devices, int calls_per_device);
 
 /*
  * What the kernels size their grids by on the current device: the number of SMs and

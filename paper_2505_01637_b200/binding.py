@@ -50,6 +50,8 @@ SIGNATURES = {
     "morello_matmul_accum_noalloc": (_int, [_int, _i64, _i64, _i64, _i64, _vp, _vp, _vp, _vp]),
     "morello_noalloc_scratch_limit": (_sz, []),
     "morello_select_path": (_int, [_i64, _i64, _i64, _i64]),
+    "morello_describe_route": (_int, [_i64, _i64, _i64, _i64, ctypes.c_char_p, _sz]),
+    "morello_selftest_per_device_once": (_int, [_int, _int]),
     "morello_matmul_accum_forced": (_int, [_int, _int, _i64, _i64, _i64, _i64, _vp, _vp, _vp,
                                            _vp, _sz, _vp]),
     "morello_workspace_bytes_forced": (_sz, [_int, _int, _i64, _i64, _i64, _i64]),
@@ -203,6 +205,17 @@ def morello_noalloc_scratch_limit() -> int:
 
 def morello_select_path(b, m, k, n) -> int:
     return int(lib().morello_select_path(b, m, k, n))
+
+
+def morello_describe_route(b, m, k, n) -> str:
+    """One line naming the kernel, tile and k slices the selector picks for this shape."""
+    buf = ctypes.create_string_buffer(512)
+    _check(lib().morello_describe_route(b, m, k, n, buf, len(buf)), "morello_describe_route")
+    return buf.value.decode()
+
+
+def morello_selftest_per_device_once(devices, calls_per_device) -> int:
+    return int(lib().morello_selftest_per_device_once(devices, calls_per_device))
 
 
 def morello_matmul_accum_forced(path, split_k, b, m, k, n, A, B, C, workspace=None,

@@ -2,6 +2,8 @@
 // selector and the dispatch to the two kernel families.
 #include <algorithm>
 #include <atomic>
+#include <cstdarg>
+#include <cstdio>
 #include <mutex>
 
 #include "../../include/morello.h"
@@ -36,6 +38,18 @@ int cuda_fail(cudaError_t e) {
   return MORELLO_ERR_CUDA;
 }
 
+// The library-owned buffers grow by freeing and allocating, which is illegal while `stream` is
+// being captured into a graph (it would invalidate the capture): such a call is refused
+// instead, before anything touches the device.
+bool capturing(cudaStream_t stream) {
+  cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(stream, &st) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return false;
+  }
+  return st != cudaStreamCaptureStatusNone;
+}
+
 // One-time set-up per device, under g_mutex.
 int device_state(DeviceState** out) {
   int dev = 0;
@@ -64,6 +78,20 @@ int device_state(DeviceState** out) {
   return st.status_code;
 }
 
+// Bounded text output for morello_describe_route.
+struct TextOut {
+  char* text;
+  size_t bytes, at;
+  __attribute__((format(printf, 2, 3))) void append(const char* fmt, ...) {
+    if (at + 1 >= bytes) return;
+    va_list ap;
+    va_start(ap, fmt);
+    const int w = vsnprintf(text + at, bytes - at, fmt, ap);
+    va_end(ap);
+    if (w > 0) at = std::min(bytes - 1, at + (size_t)w);
+  }
+};
+
 bool mul_overflows(int64_t a, int64_t b, int64_t* out) {
   return __builtin_mul_overflow(a, b, out);
 }
@@ -90,13 +118,10 @@ int validate(int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const vo
   return MORELLO_OK;
 }
 
-// Measured on the 2048 x 16384 weight shape (us per call, FMA kernels / tensor path):
-// m = 1: 10.98 / 11.26, m = 2: 11.79 / 11.38, m = 4: 16.6 / 11.4, m = 8: 35.6 / 11.5,
-// m = 16: 84.8 / 11.7.  Every extra row costs the FMA kernels one FMA per element of B
-// while the tensor cores take the rows for free, so the FMA kernels keep the single row (the
-// GEMV proper) and whatever the TMA engine cannot address.  Few columns do not change that:
-// 16 x 4096 x 4096 takes 80 us on the FMA kernel and 14 us on the tensor path, which cuts a
-// long k into slices of its own when the columns alone cannot occupy the device.
+// Every extra row costs the FMA kernels one FMA per element of B while the tensor cores take
+// the rows for free, so the FMA kernels keep the single row (the GEMV proper) and whatever the
+// TMA engine cannot address; from two rows on the tensor path wins, few columns included (it
+// cuts a long k into slices of its own when the columns alone cannot occupy the device).
 constexpr int kFmaMaxRows = 1;
 int select_path(int sms, int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const void* B,
                 const void* C) {
@@ -104,13 +129,9 @@ int select_path(int sms, int64_t b, int64_t m, int64_t k, int64_t n, const void*
   if (m <= kFmaMaxRows) {
     // The single row.  The FMA GEMV kernel is at its best when its 64-column strips (times its
     // k slices) fill the two block slots per SM exactly once and k is short; elsewhere the
-    // operand-swapped tensor kernel streams B faster (128-column strips, deeper ring).
-    // Measured, us per call, FMA GEMV / operand-swapped, k x n: 2048 x 8192: 8.2 / 9.2; 2048 x
-    // 16384: 11.1 / 11.5; 4096 x 8192: 12.3 / 13.8; 8192 x 8192: 22.7 / 23.3; but 2048 x 12288
-    // (384 blocks): 13.9 / 9.9; 2048 x 20480: 19.1 / 14.0; 4096 x 32000: 45.9 / 40.0; 4096 x
-    // 16384: 21.6 / 20.8; 8192 x 16384: 41.3 / 39.3; 4096 x 65536: 87.2 / 81.3.
-    // (Below 16 MB of B both finish within a launch latency or two; the FMA kernels are the
-    // lighter launch: 2048 x 2048: 4.7 / 5.4.)
+    // operand-swapped tensor kernel streams B faster (128-column strips, deeper ring).  Below
+    // 16 MB of B both finish within a launch latency or two and the FMA kernels are the lighter
+    // launch.
     if (b > 65535 || b * k * n < (1ll << 23) || !stream_shape_supported(b, 1, k, n, B))
       return MORELLO_PATH_SKINNY;
     const StreamPlan pl = stream_plan(sms, b, 1, k, n, 0);
@@ -124,13 +145,11 @@ int select_path(int sms, int64_t b, int64_t m, int64_t k, int64_t n, const void*
 }
 
 // Extents the TMA engine cannot address (k % 8 != 0 or n % 8 != 0): the FMA kernels take the
-// rows in chunks of 16 and stream B once per chunk, the padded-copy route pays one pass over A
-// and B, one over C and a handful of launches and then runs at tensor-core speed.  Measured
-// (us per call, FMA kernels with narrow loads / padded copies): 512 x 1000 x 1001: 723 / 16.5, 2048 x 2047 x
-// 2049: 9,380 / 48.6, 4096 x 4095 x 4097: 54,352 / 189, 16 x 2048 x 16383: 258 / 48.8, 64 x
-// 1001 x 1001: 91 / 18.5; 17 x 100 x 100 (two chunks): 10.9 on the FMA kernels.
-// Estimated cost of both, in microseconds; pointers that are merely misaligned keep the FMA
-// route (the workspace a shape may need must not depend on them).
+// rows in chunks of 16 and stream B once per chunk; the padded-copy route pays one pass over the
+// operands that need a copy and a launch or two more, and then runs at tensor-core speed.
+// Estimated cost of both, in microseconds (the constants are fits to measurements on a B200);
+// pointers that are merely misaligned keep the FMA route (the workspace a shape may need must
+// not depend on them).
 bool staged_wins(int64_t b, int64_t m, int64_t k, int64_t n) {
   if ((k % 8 == 0 && n % 8 == 0) || m < 2) return false;
   const int64_t limit = (1ll << 31) - 8;   // tensor-map extents are 32-bit
@@ -138,8 +157,7 @@ bool staged_wins(int64_t b, int64_t m, int64_t k, int64_t n) {
   const double bytes_a = 2.0 * b * m * k, bytes_b = 2.0 * b * k * n, bytes_c = 4.0 * b * m * n;
   // The FMA kernel's cost per MB of B for a chunk of r rows: bound by memory up to a few rows,
   // then by one FMA per row and element.  Its flat form reads unaligned rows in aligned
-  // 16-byte granules (measured on 2048 x 16383, us per call: 1 row 16.6, 2: 19.6, 4: 24.6,
-  // 8: 37.1, 16: 79.1); tiny shapes fall back to narrow loads, which cost more of both.
+  // 16-byte granules; tiny shapes fall back to narrow loads, which cost more of both.
   const bool flat = k >= 64 && n >= 16;
   const int vec = n % 8 == 0 ? 8 : n % 4 == 0 ? 4 : n % 2 == 0 ? 2 : 1;
   const double base = flat ? 0.25 : vec == 8 ? 0.2 : vec == 4 ? 0.3 : vec == 2 ? 0.37 : 0.5;
@@ -278,6 +296,7 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     if (own_scratch) {
       std::lock_guard<std::mutex> lock(g_mutex);
       if (st->scratch_bytes < need) {
+        if (capturing(static_cast<cudaStream_t>(stream))) return MORELLO_ERR_WORKSPACE;
         // Work already enqueued may still be using the old buffer.
         cudaError_t e = cudaDeviceSynchronize();
         if (e != cudaSuccess) return cuda_fail(e);
@@ -348,6 +367,10 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
 }
 
 }  // namespace
+
+void count_launches(uint64_t launches) { g_launches.fetch_add(launches, std::memory_order_relaxed); }
+int record_cuda_error(cudaError_t e) { return cuda_fail(e); }
+
 }  // namespace morello
 
 using namespace morello;
@@ -482,6 +505,7 @@ int run_f32(int64_t b, int64_t m, int64_t k, int64_t n, const float* A, const fl
   {
     std::lock_guard<std::mutex> lock(g_mutex);
     if (st->split_bytes < need) {
+      if (capturing(static_cast<cudaStream_t>(stream))) return MORELLO_ERR_WORKSPACE;
       cudaError_t e = cudaDeviceSynchronize();   // work in flight may still read the old buffer
       if (e != cudaSuccess) return cuda_fail(e);
       if (st->split) cudaFree(st->split);
@@ -548,6 +572,10 @@ int morello_matmul_accum_host(int64_t b, int64_t m, int64_t k, int64_t n, const 
                c_bytes = (size_t)b * m * n * 4;
   const size_t need = round256(a_bytes) + round256(b_bytes) + round256(c_bytes);
   cudaError_t e;
+  // One staging buffer per device: host threads take turns for the whole call (it is synchronous
+  // anyway), so that neither the copies nor a regrowth of the buffer can cross another call.
+  static std::mutex host_mutex;
+  std::lock_guard<std::mutex> whole_call(host_mutex);
   {
     std::lock_guard<std::mutex> lock(g_mutex);
     if (st->stage_bytes < need) {
@@ -597,6 +625,71 @@ int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n) {
   return select_path(sms, b, m, k, n, fake, fake, fake);
 }
 
+int morello_describe_route(int64_t b, int64_t m, int64_t k, int64_t n, char* text, size_t text_bytes) {
+  if (!text || text_bytes == 0) return MORELLO_ERR_NULL_POINTER;
+  text[0] = 0;
+  bool empty = false;
+  const void* fake = reinterpret_cast<const void*>(uintptr_t(4096));   // 16-byte-aligned operands
+  const int rc = validate(b, m, k, n, fake, fake, fake, &empty);
+  if (rc != MORELLO_OK) return rc;
+  if (empty) {
+    snprintf(text, text_bytes, "nothing to launch (an empty sum)");
+    return MORELLO_OK;
+  }
+  int sms = 148;   // without a usable device, a B200's
+  DeviceState* st = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (device_state(&st) == MORELLO_OK) sms = st->info.sms;
+  }
+  TextOut out{text, text_bytes, 0};
+#define put(...) out.append(__VA_ARGS__)
+  int64_t kk = k, nn = n;
+  const bool staged = staged_wins(b, m, k, n);
+  if (staged) {
+    const PadPlan pp = pad_plan(b, m, k, n, fake, fake, fake);
+    kk = pp.k8;
+    nn = pp.n8;
+    put("padded copies of%s%s%s to k=%lld n=%lld, then ", pp.stage_a ? " A" : "", pp.stage_b ? " B" : "",
+        pp.stage_c ? " C" : "", (long long)kk, (long long)nn);
+  }
+  const int path = staged ? MORELLO_PATH_TCGEN05 : select_path(sms, b, m, k, n, fake, fake, fake);
+  if (path == MORELLO_PATH_TCGEN05) {
+    const GemmPlan pl = gemm_plan(sms, b, m, kk, nn, 0);
+    if (!pl.supported) return MORELLO_ERR_UNSUPPORTED_PATH;
+    if (pl.form == 3) {
+      put("tcgen05 swap_kernel: operands swapped, strips of 128 columns, %d rows of A per MMA", pl.tile_n);
+      if (pl.split_k > 1) put(", %d k slices added inside a cluster", pl.split_k);
+    } else {
+      put("tcgen05 gemm_kernel: %s per %d x %d tile", pl.form == 2 ? "a CTA pair" : "one CTA",
+          pl.form == 2 ? 256 : 128, pl.tile_n);
+      const int64_t tile_m = pl.form == 2 ? 256 : 128;
+      const int64_t tiles = b * ((m + tile_m - 1) / tile_m) * ((nn + pl.tile_n - 1) / pl.tile_n);
+      const int64_t units = std::max(1, pl.form == 2 ? gemm_pair_units(sms) : sms);
+      const int64_t tail = tiles % units;
+      if (pl.halves && pl.ws_split <= 1 && (pl.tile_n / (pl.form == 2 ? 2 : 1) / 2) % 64 == 0 && tiles > units &&
+          tail > 0 && 2 * tail <= units)
+        put(", the %lld tiles of the last wave cut into column halves", (long long)tail);
+    }
+    if (pl.ws_split > 1) put(", %d k slices through the workspace + reduce launch", pl.ws_split);
+  } else {
+    const int which = skinny_kernel_for(0, b, m, k, n, fake);
+    if (which == SKINNY_STREAM) {
+      const StreamPlan pl = stream_plan(sms, b, (int)m, k, n, 0);
+      put("fma gemv_stream_kernel: TMA ring, %d strips of 64 columns x %d k slices%s", pl.strips, pl.split_k,
+          pl.split_k > 1 ? (pl.cluster_k ? " added inside a cluster" : " + reduce launch") : "");
+    } else {
+      const int rows = (int)std::min<int64_t>(kSkinnyMaxRows, m);
+      const SkinnyPlan pl = skinny_plan(sms, b, rows, k, n, skinny_vec(n, fake), 0);
+      put("fma skinny_kernel: register streaming%s, %lld chunk%s of <= 16 rows, %d-element loads, %d column blocks x %d k slices%s",
+          pl.flat ? " (aligned granules, shifted columns)" : "", (long long)((m + kSkinnyMaxRows - 1) / kSkinnyMaxRows),
+          m > kSkinnyMaxRows ? "s" : "", pl.vec, pl.col_blocks, pl.split_k, pl.split_k > 1 ? " + reduce launch" : "");
+    }
+  }
+#undef put
+  return MORELLO_OK;
+}
+
 int morello_read_device_status(void* stream, uint32_t* detail) {
   if (detail) *detail = 0;
   DeviceState* st = nullptr;
@@ -639,6 +732,20 @@ int morello_selftest_wait_timeout(uint32_t limit_ms, void* stream) {
   int verdict = 0;
   if ((e = cudaMemcpy(&verdict, gave_up, 4, cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(e);
   return verdict == 1 ? MORELLO_OK : MORELLO_ERR_CUDA;
+}
+
+int morello_selftest_per_device_once(int devices, int calls_per_device) {
+  if (devices < 0 || calls_per_device < 0) return -1;
+  PerDeviceOnce once;
+  int runs = 0;
+  for (int c = 0; c < calls_per_device; ++c)
+    for (int d = 0; d < devices; ++d)
+      // A first attempt that fails is not remembered: device 1's set-up fails once, then works.
+      (void)once.run(d, [&] {
+        ++runs;
+        return (d == 1 && runs <= devices) ? cudaErrorInvalidValue : cudaSuccess;
+      });
+  return runs;
 }
 
 int morello_device_limits(int* sms, int* cta_pairs) {

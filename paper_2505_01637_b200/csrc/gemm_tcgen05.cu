@@ -432,23 +432,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 // blocks of B into L2 (nothing reaches the SM, so this is legal early), and a block lets
 // dependents launch once its producer has issued its last load.  With more rows a stage
 // carries more of A and the same budget would hold too little of B in flight: the ring then
-// takes 200 KiB and the next call's block follows when this one leaves (measured, 2048 x
-// 16384, 108 / 200 KiB: 32 rows 12.9 / 12.6 us, 48 rows 14.8 / 13.1, 64 rows 15.4 / 13.8).
-#ifndef MORELLO_SWAP_RING_KIB
-#define MORELLO_SWAP_RING_KIB 108        // stages of the <= 16-row kernel: two blocks fit an SM
-#endif
-#ifndef MORELLO_SWAP_BIG_RING_KIB
-#define MORELLO_SWAP_BIG_RING_KIB 200    // stages with more rows of A
-#endif
-#ifndef MORELLO_SWAP_PREFETCH_BLOCKS
-#define MORELLO_SWAP_PREFETCH_BLOCKS 6
-#endif
+// takes 200 KiB and the next call's block follows when this one leaves.
+constexpr int kSwapRingKiB = 108;        // stages of the <= 16-row kernel: two blocks fit an SM
+constexpr int kSwapBigRingKiB = 200;     // stages with more rows of A
 template <int kRowsA>
 struct SwapShape {
   static constexpr int kBytesStrip = 2 * kBoxBytesB;                  // 128 columns x 64 k: 16 KiB
   static constexpr int kBytesRows = kRowsA * kTileK * 2;              // 2 .. 8 KiB
   static constexpr int kStageBytes = kBytesStrip + kBytesRows;
-  static constexpr int kRingKiB = kRowsA <= 16 ? MORELLO_SWAP_RING_KIB : MORELLO_SWAP_BIG_RING_KIB;
+  static constexpr int kRingKiB = kRowsA <= 16 ? kSwapRingKiB : kSwapBigRingKiB;
   static constexpr int kFit = (kRingKiB * 1024) / kStageBytes;
   static constexpr int kStages = kFit < kMaxStages ? kFit : kMaxStages;
   static constexpr int kTmemCols = kRowsA <= 32 ? 32 : 64;
@@ -457,7 +449,7 @@ struct SwapShape {
 };
 constexpr int kSwapStripCols = 128;
 constexpr int kSwapMaxRows = 64;
-constexpr int kSwapPrefetchBlocks = MORELLO_SWAP_PREFETCH_BLOCKS;   // k blocks asked into L2 before the wait
+constexpr int kSwapPrefetchBlocks = 6;   // k blocks asked into L2 before the wait
 
 struct SwapParams {
   float* C;
@@ -497,8 +489,7 @@ struct SwapBarriers {
 // blockIdx.x, blockIdx.x + gridDim.x, ...; its producer keeps the stage ring full across items,
 // so the loads of the next items run under the epilogue of the current one.  With many short
 // items (batched problems with a short k) that removes the per-block set-up from the critical
-// path (256 x 1 x 128 x 4096: 71.8 us with one block per item).  With one item per block (the
-// long streams the kernel was tuned on) nothing changes.
+// path.  With one item per block (the long streams the kernel was tuned on) nothing changes.
 template <int kRowsA, bool kClusterK, bool kPersistent>
 __global__ void __launch_bounds__(kThreads)
 swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -824,13 +815,11 @@ namespace {
 
 template <bool kPair, int kTileN>
 cudaError_t set_smem_attribute() {
-  static std::once_flag once;
-  static cudaError_t err = cudaSuccess;
-  std::call_once(once, [] {
-    err = cudaFuncSetAttribute(gemm_kernel<kPair, kTileN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)Shape<kPair, kTileN>::kSmemBytes);
+  static PerDeviceOnce once;   // the attribute belongs to the current device's copy of the kernel
+  return once.run_current([] {
+    return cudaFuncSetAttribute(gemm_kernel<kPair, kTileN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)Shape<kPair, kTileN>::kSmemBytes);
   });
-  return err;
 }
 
 // How many CTA pairs the device can hold at once.  A pair needs two SMs of one
@@ -889,8 +878,7 @@ int gemm_pair_units(int sms) { return pair_units(sms); }
 // Few tiles and a long k: a call whose tiles fill less than half the device is cut along k as
 // well.  Each (tile, slice) item stores its sums to partial[slice][b][m][n] in the workspace
 // and one more launch adds the slices in slice order, then C -- the bits do not depend on which
-// block finished first.  (Measured, us per call before / after: 64 x 16384 x 2048: 46.5; 128 x
-// 16384 x 2048: 52.8; 512 x 16384 x 2048: 53.8.)
+// block finished first.
 namespace {
 
 constexpr int kWsMaxSplit = 8;
@@ -930,12 +918,9 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob
     const int64_t want = std::min<int64_t>(units / tiles, k_blocks / kWsMinBlocks);
     return ws_fit((int)std::min<int64_t>(want, kWsMaxSplit), k_blocks, b, m, n);
   };
-  // Form 3: the operand-swapped kernel.  By shape it takes every call of at most 64 rows
-  // (measured on 2048 x 16384, us per call, swapped / 128-row tiles: m = 16: 11.7 / 14.2, 32:
-  // 12.6 / 14.4, 48: 13.1 / 14.6, 64: 13.8 / 14.9; with few columns it wins as well: 16 x 4096 x
-  // 4096: 14.4 / 16.0).  Beyond 64 rows the 128-row tiles win: an accumulator of more than 64
-  // columns per thread cannot be paired with an early read of C in registers, and sending the
-  // sums out as L2 reductions instead cost more than it saved (96 rows: 16.7 against 15.4 us).
+  // Form 3: the operand-swapped kernel.  By shape it takes every call of at most 64 rows.
+  // Beyond 64 rows the 128-row tiles win: an accumulator of more than 64 columns per thread
+  // cannot be paired with an early read of C in registers.
   if (form == 3 || (form == 0 && tile_n == 0 && m <= kSwapMaxRows)) {
     // With form 3 the knob's column field is the number of k slices instead (0 = by shape).
     const int forced_split = tile_n / 64;
@@ -945,12 +930,10 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob
     const int64_t strips = b * ((n + kSwapStripCols - 1) / kSwapStripCols);
     int split = forced_split;
     if (split == 0) {
-      // Few strips and a long k: cut k.  Measured (us per call, 1 / 2 / 4 / 8 slices): 16 rows,
-      // 16 strips (16384 x 2048): 48 / 31 / 19 / 15; 32 strips (4096 x 4096): 14.4 / 13.4 / 11.1 /
-      // 10.3; 64 strips (4096 x 8192): 15.6 / 16.5; 128 strips (2048 x 16384): 11.8 / 15.9.  With
-      // more than 16 rows a block fills an SM and clusters of them pack badly (48 rows, 16
-      // strips: 14.2 / 24.1 / 19.3).  So: up to 16 rows and up to 32 strips, as many slices as
-      // leave four k blocks each; the other shapes of few strips go through the workspace.
+      // Few strips and a long k: cut k inside a cluster.  That pays up to 16 rows and up to 32
+      // strips (with more rows a block fills an SM and clusters of such blocks pack badly; with
+      // more strips the device is busy anyway): as many slices as leave eight k blocks each.  The
+      // other shapes of few strips go through the workspace.
       split = 1;
       if (forced_ws <= 1 && a_box_rows(m) == 16 && strips <= 32 && b <= 65535)
         while (split < 8 && k_blocks >= 8 * split) split *= 2;
@@ -964,9 +947,8 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob
       (form == 2 && tile_n == 64))
     return GemmPlan{false, 0, 0, 0, false, 1, 1};
   if (form != 2 && tile_n == 0 && m <= kRowsPerCta) {
-    // First without k slices (they cost a second launch and a trip through the workspace:
-    // 128 x 2048 x 16384 runs 15.4 us on 128 tiles of 128 columns, 23.1 us on 64 tiles of 256
-    // columns cut in two); with them only when even 64-column tiles leave the device idle.
+    // First without k slices (they cost a second launch and a trip through the workspace); with
+    // them only when even 64-column tiles leave the device idle.
     for (int tn = 256; tn >= 64; tn >>= 1) {
       const int64_t tiles = b * ((n + tn - 1) / tn);
       if (tiles * 5 >= (int64_t)sms * 4 && forced_ws <= 1) return finish(GemmPlan{true, 1, tn, 0, halves, 1, 1});
@@ -1091,11 +1073,10 @@ cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_
                              const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
                              bool overwrite, int bt, const KSegments* seg, cudaStream_t stream) {
   using S = SwapShape<kRowsA>;
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(swap_kernel<kRowsA, kClusterK, kPersistent>,
-                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::kSmemBytes);
+  static PerDeviceOnce once;   // the attribute belongs to the current device's copy of the kernel
+  const cudaError_t attr_err = once.run_current([] {
+    return cudaFuncSetAttribute(swap_kernel<kRowsA, kClusterK, kPersistent>,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)S::kSmemBytes);
   });
   if (attr_err != cudaSuccess) return attr_err;
   SwapParams p{};

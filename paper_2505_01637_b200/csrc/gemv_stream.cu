@@ -44,38 +44,22 @@ namespace {
 
 using namespace sm100;
 
-// Tunables (compile-time; the defaults are the measured best for 1 x 2048 x 16384).
-#ifndef MORELLO_GEMV_STRIP_COLS
-#define MORELLO_GEMV_STRIP_COLS 64
-#endif
-#ifndef MORELLO_GEMV_STAGES
-#define MORELLO_GEMV_STAGES 5
-#endif
-#ifndef MORELLO_GEMV_PREFETCH_BOXES
-#define MORELLO_GEMV_PREFETCH_BOXES 6
-#endif
-constexpr int kStripCols = MORELLO_GEMV_STRIP_COLS;         // columns per thread block: 64 or 128
-#ifndef MORELLO_GEMV_BOX_ROWS
-#define MORELLO_GEMV_BOX_ROWS 128
-#endif
-#ifndef MORELLO_GEMV_FFMA2
-#define MORELLO_GEMV_FFMA2 1
-#endif
-constexpr int kBoxRows = MORELLO_GEMV_BOX_ROWS;             // k rows per stage: 64 or 128
-constexpr int kStageBytes = kBoxRows * kStripCols * 2;      // 8 or 16 KiB
-constexpr int kStages = MORELLO_GEMV_STAGES;
+// Geometry (the measured best for 1 x 2048 x 16384).
+constexpr int kStripCols = 64;                              // columns per thread block
+constexpr int kBoxRows = 128;                               // k rows per stage
+constexpr int kStageBytes = kBoxRows * kStripCols * 2;      // 16 KiB
+constexpr int kStages = 5;
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumers = 32 * kConsumerWarps;
 constexpr int kThreads = 32 + kConsumers;
 constexpr int kMaxSliceBytes = 32 * 1024;                   // bf16 rows of A staged per block
 constexpr int max_slice_k(int m_tile) { return kMaxSliceBytes / (2 * m_tile); }
 constexpr int kMaxClusterK = 8;                             // k slices added inside one cluster
-constexpr int kPrefetchBoxes = MORELLO_GEMV_PREFETCH_BOXES; // boxes asked into L2 before the wait
+constexpr int kPrefetchBoxes = 6;                           // boxes asked into L2 before the wait
 constexpr int kLanesPerRow = kStripCols / 8;                // 16-byte chunks per box row
 constexpr int kRowsPerWarp = 32 / kLanesPerRow;             // box rows one warp-wide load covers
 constexpr int kRowsPerPass = kRowsPerWarp * kConsumerWarps;
 constexpr int kPasses = kBoxRows / kRowsPerPass;
-static_assert(kStripCols == 64 || kStripCols == 128, "strip width");
 
 struct StreamParams {
   const uint16_t* A;
@@ -119,13 +103,7 @@ __device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
   asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
 }
 __device__ __forceinline__ void fma2(uint64_t& acc, uint64_t a, uint64_t b) {
-#if MORELLO_GEMV_FFMA2
   asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
-#else
-  float a0, a1, b0, b1, c0, c1;
-  unpack2(a, a0, a1); unpack2(b, b0, b1); unpack2(acc, c0, c1);
-  acc = pack2(fmaf(a0, b0, c0), fmaf(a1, b1, c1));
-#endif
 }
 
 template <int M_T, bool kClusterK>
@@ -397,8 +375,7 @@ cudaError_t get_b_map(const BKey& key, CUtensorMap* out) {
   cudaError_t err = make_tensor_map_3d(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, key.b,
                                        (uint64_t)key.n, (uint64_t)key.k, (uint64_t)key.bsz,
                                        kStripCols, kBoxRows, CU_TENSOR_MAP_SWIZZLE_NONE,
-                                       kStripCols == 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B
-                                                        : CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+                                       CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
   if (err != cudaSuccess) return err;
   e.stamp = ++g_bstamp;
   e.valid = true;
@@ -416,11 +393,10 @@ template <int M_T, bool kClusterK>
 cudaError_t launch(const StreamPlan& plan, const CUtensorMap& map, const StreamParams& prm,
                    int64_t b, cudaStream_t stream) {
   auto kern = gemv_stream_kernel<M_T, kClusterK>;
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [&] {
-    attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)smem_for(M_T, max_slice_k(M_T)));
+  static PerDeviceOnce once;   // the attribute belongs to the current device's copy of the kernel
+  const cudaError_t attr_err = once.run_current([&] {
+    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)smem_for(M_T, max_slice_k(M_T)));
   });
   if (attr_err != cudaSuccess) return attr_err;
   cudaLaunchConfig_t cfg{};

@@ -8,7 +8,40 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <mutex>
+
 namespace morello {
+
+// Set-up that has to happen once per device and not once per process: a kernel's function
+// attributes (the opt-in to more than 48 KiB of dynamic shared memory, say) belong to the
+// current device's copy of the kernel.  run(dev, fn) calls fn() the first time it sees device
+// `dev` and hands back its result; a failure is not remembered, the next call tries again.
+// Devices beyond the table run fn() every time (a cheap host call).
+class PerDeviceOnce {
+ public:
+  static constexpr int kSlots = 64;
+  template <typename F>
+  cudaError_t run(int dev, F&& fn) {
+    if (dev < 0 || dev >= kSlots) return fn();
+    std::lock_guard<std::mutex> lock(mutex_);
+    if (done_[dev]) return cudaSuccess;
+    const cudaError_t e = fn();
+    done_[dev] = (e == cudaSuccess);
+    return e;
+  }
+  // The same, for the device that is current on the calling thread.
+  template <typename F>
+  cudaError_t run_current(F&& fn) {
+    int dev = -1;
+    const cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    return run(dev, static_cast<F&&>(fn));
+  }
+
+ private:
+  std::mutex mutex_;
+  bool done_[kSlots] = {};
+};
 
 // Device-side status word written by bounded waits that gave up.
 // 0 = OK; otherwise (site << 16) | detail, first writer wins.
@@ -148,6 +181,13 @@ cudaError_t colmajor_fallback_launch(int64_t b, int64_t m, int64_t k, int64_t n,
 cudaError_t packed_fallback_launch(int64_t strip, int64_t b, int64_t m, int64_t k, int64_t n,
                                    const uint16_t* A, const uint16_t* Bp, float* C, bool overwrite,
                                    cudaStream_t stream, uint64_t* launches);
+
+// ---- bookkeeping shared with the other translation units' entry points (api.cu) ----------
+// Adds to the count morello_launch_count() reports.
+void count_launches(uint64_t launches);
+// Records a failed CUDA call where morello_last_cuda_error() finds it, clears the runtime's
+// sticky error and returns MORELLO_ERR_CUDA.
+int record_cuda_error(cudaError_t e);
 
 // ---- self-test of the bounded device-side waits --------------------------------
 // One thread waits at most limit_ns on a barrier nothing arrives on, gives up, records the

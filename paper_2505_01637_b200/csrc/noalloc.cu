@@ -38,25 +38,24 @@ std::mutex g_noalloc_mutex;
 // resolves the device address of the static array.  No allocation.
 int noalloc_device(NoAllocDevice** out) {
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return MORELLO_ERR_CUDA;
+  cudaError_t ce = cudaGetDevice(&dev);
+  if (ce != cudaSuccess) return record_cuda_error(ce);
   if (dev < 0 || dev >= kMaxDevices) return MORELLO_ERR_UNSUPPORTED_DEVICE;
   std::lock_guard<std::mutex> lock(g_noalloc_mutex);
   NoAllocDevice& st = g_noalloc[dev];
   if (!st.ready) {
     int major = 0, sms = 0;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-      return MORELLO_ERR_CUDA;
+    if ((ce = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev)) != cudaSuccess ||
+        (ce = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+      return record_cuda_error(ce);
     st.sms = sms;
     if (major != 10) {
       st.status = MORELLO_ERR_UNSUPPORTED_DEVICE;
     } else {
       void* ptr = nullptr;
       const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
-      if (e != cudaSuccess || ptr == nullptr) {
-        (void)cudaGetLastError();
-        return MORELLO_ERR_CUDA;  // not latched: a later call may try again
-      }
+      if (e != cudaSuccess || ptr == nullptr)   // not latched: a later call may try again
+        return record_cuda_error(e != cudaSuccess ? e : cudaErrorInvalidSymbol);
       st.scratch = static_cast<float*>(ptr);
       st.status = MORELLO_OK;
     }
@@ -113,10 +112,11 @@ int morello_matmul_accum_noalloc(int split_k, int64_t b, int64_t m, int64_t k, i
         skinny_launch(plan, b, mc, k, n, a + i0 * k, m * k, static_cast<const uint16_t*>(B),
                       C + i0 * n, m * n, st->scratch, static_cast<cudaStream_t>(stream), &launches);
     if (e != cudaSuccess) {
-      (void)cudaGetLastError();
-      return MORELLO_ERR_CUDA;
+      count_launches(launches);
+      return record_cuda_error(e);
     }
   }
+  count_launches(launches);
   return MORELLO_OK;
 }
 

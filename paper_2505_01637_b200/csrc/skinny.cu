@@ -419,9 +419,8 @@ SkinnyPlan plan_impl(int sms, int64_t b, int m, int64_t k, int64_t n, int vec, i
   pl.k_per_split = kps;
   pl.split_k = (int)((std::max<int64_t>(k, 1) + kps - 1) / kps);
   // More thread blocks than SMs with a single row: blocks of 512 threads, so that two share an
-  // SM instead of running in two rounds (1 x 4096 x 32001: 55.3 -> 44 us, 1 x 768 x 50257:
-  // 25.6 -> 20 us; with one block per SM the full 1024 threads are better: 1 x 2048 x 16383:
-  // 16.6 against 19.1 us).
+  // SM instead of running in two rounds (with at most one block per SM the full 1024 threads
+  // are better).
   if (pl.m_tile == 1 && blocks * pl.split_k > sms) max_threads = std::min(max_threads, 512);
   // Row lanes: as many as the thread budget allows, a multiple of 8 when possible,
   // never more than the slice has rows.

@@ -79,6 +79,37 @@ def test_selector_is_shape_based(mb):
     assert mb.morello_select_path(1, -1, 4, 4) == -1
 
 
+def test_route_description_names_the_kernel(mb):
+    d = mb.morello_describe_route
+    assert d(1, 1, 2048, 16384).startswith("fma gemv_stream_kernel")          # the headline GEMV
+    assert "256 strips" in d(1, 1, 2048, 16384)
+    assert d(1, 16, 2048, 16384).startswith("tcgen05 swap_kernel")            # operands swapped
+    assert "16 rows" in d(1, 16, 2048, 16384)
+    assert "a CTA pair per 256 x 256 tile" in d(1, 4096, 4096, 4096)
+    assert "one CTA per 128 x" in d(1, 128, 2048, 16384)
+    assert "k slices through the workspace" in d(1, 512, 16384, 2048)
+    assert "added inside a cluster" in d(1, 16, 16384, 2048)
+    assert d(1, 2048, 2047, 2049).startswith("padded copies of A B C to k=2048 n=2056, then tcgen05")
+    assert d(1, 4, 4, 16).startswith("fma skinny_kernel")
+    assert "shifted columns" in d(1, 1, 2048, 16383)
+    assert d(0, 4, 4, 4).startswith("nothing to launch")
+    # a short buffer is filled up to its last byte and NUL-terminated; bad arguments are refused
+    buf = ctypes.create_string_buffer(b"x" * 12, 12)
+    assert mb.lib().morello_describe_route(1, 4096, 4096, 4096, buf, 12) == mb.MORELLO_OK
+    assert buf.raw == b"tcgen05 gem\0"
+    assert mb.lib().morello_describe_route(1, 4, 4, 4, None, 0) == mb.MORELLO_ERR_NULL_POINTER
+    assert mb.lib().morello_describe_route(1, -4, 4, 4, buf, 12) == mb.MORELLO_ERR_INVALID_SHAPE
+
+
+def test_per_device_setup_runs_once_per_device_and_retries_failures(mb):
+    once = mb.morello_selftest_per_device_once
+    assert once(1, 5) == 1          # one device, five calls: set up once
+    assert once(4, 3) == 5          # four devices: once each, plus device 1's failed first attempt
+    assert once(4, 1) == 4
+    assert once(0, 3) == 0
+    assert once(-1, 3) == -1
+
+
 def test_missing_library_fails_loudly(mb, monkeypatch):
     import importlib
     from paper_2505_01637_b200 import binding

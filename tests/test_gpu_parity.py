@@ -70,6 +70,12 @@ def test_configs_1_to_3_full(index, variant):
                what="%s/%s" % (w.CONFIGS[index].name, variant))
 
 
+@pytest.mark.parametrize("variant", ["random", "integer"])
+def test_config_4_whole_output(variant):
+    A, B, C = w.make_config(3, variant)
+    check_full(A, B, C, integer=(variant != "random"), what="%s/%s" % (w.CONFIGS[3].name, variant))
+
+
 @pytest.mark.parametrize("index", [3, 4])
 @pytest.mark.parametrize("variant", ["random", "integer"])
 def test_configs_4_and_5_sampled_rows(index, variant):

@@ -6,6 +6,8 @@ import os
 import subprocess
 import sys
 
+import pytest
+
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 WORKER = r"""
@@ -68,3 +70,33 @@ def test_reference_arm_prints_on_rank_zero_only():
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
     assert line["unit"] == "GB/s" and line["higher_is_better"] is True
+
+
+def test_gpus_n_without_a_launcher_environment_starts_the_ranks_itself():
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.rank_command(2, ["--gpus", "2", "--steps", "3"])
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node" in cmd
+    assert cmd[cmd.index("--nproc-per-node") + 1] == "2" and cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-4:] == ["--gpus", "2", "--steps", "3"] and cmd[-5].endswith("bench.py")
+    # end to end on CPU through the reference arm: two ranks are started, rank 0 alone prints
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE")}
+    run = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                          "--steps", "2", "--warmup", "1"], env=env, capture_output=True, text=True, timeout=900)
+    assert run.returncode == 0, run.stderr[-2000:]
+    lines = [l for l in run.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2
+
+
+def test_loop_count_and_spread():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.loop_count(0.25e-3) == 200            # 20 steps of 12.5 us: 200 loops make 50 ms
+    assert bench.loop_count(1.0) == bench.MIN_LOOPS      # long loops: the minimum number of repeats
+    assert bench.loop_count(1e-9) == bench.MAX_LOOPS
+    s = bench.spread([2e-4, 1e-4, 4e-4], 10)
+    assert s["us_per_step_median"] == pytest.approx(20.0) and s["us_per_step_min"] == pytest.approx(10.0)
+    assert s["us_per_step_max"] == pytest.approx(40.0) and s["loops"] == 3
+    assert bench.workload_name(bench.w.CONFIGS[1]).startswith("cfg2_gemv b,m,k,n=[1, 1, 2048, 16384]")
