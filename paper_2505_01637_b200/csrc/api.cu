@@ -167,7 +167,7 @@ bool staged_wins(int64_t b, int64_t m, int64_t k, int64_t n) {
   double fma = (double)full_chunks * (5.0 + mb_b * std::max(base, 16 * per_row));
   if (rest) fma += 5.0 + mb_b * std::max(base, (double)rest * per_row);
   // Copies in and out, then the tensor-core call itself: its FLOPs or its pass over memory.
-  const double staged = 14.0 + (2.0 * (bytes_a + bytes_b) + 3.0 * bytes_c) / 4.4e6 +
+  const double staged = 9.0 + (2.0 * (bytes_a + bytes_b) + 0.5 * bytes_c) / 4.4e6 +
                         std::max(2.0 * b * m * k * n / 1e9, (bytes_a + bytes_b + 2.0 * bytes_c) / 6e6);
   return staged < fma;
 }
@@ -177,7 +177,7 @@ bool staged_wins(int64_t b, int64_t m, int64_t k, int64_t n) {
 size_t staged_workspace(int sms, int64_t b, int64_t m, int64_t k, int64_t n) {
   const void* odd = reinterpret_cast<const void*>(uintptr_t(4100));   // 4-byte aligned only
   const PadPlan pp = pad_plan(b, m, k, n, odd, odd, odd);
-  return pp.bytes_a + pp.bytes_b + pp.bytes_c + gemm_plan(sms, b, m, pp.k8, pp.n8, 0).workspace_bytes;
+  return pp.bytes_a + pp.bytes_b + gemm_plan(sms, b, m, pp.k8, pp.n8, 0).workspace_bytes;
 }
 
 // The knob of the forced entry point on the skinny path: knob % 1024 is the split of the k
@@ -289,7 +289,7 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     pad_gemm = gemm_plan(sms, b, m, pad.k8, pad.n8, 0);
     if (!pad_gemm.supported) return MORELLO_ERR_UNSUPPORTED_PATH;
   }
-  const size_t need = staged ? pad.bytes_a + pad.bytes_b + pad.bytes_c + pad_gemm.workspace_bytes
+  const size_t need = staged ? pad.bytes_a + pad.bytes_b + pad_gemm.workspace_bytes
                       : bt_fallback ? 0 : workspace_for(sms, path, split_k, b, m, k, n, B);
   float* ws = static_cast<float*>(workspace);
   if (need > 0) {
@@ -323,18 +323,15 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
     char* base = reinterpret_cast<char*>(ws);
     uint16_t* a_pad = reinterpret_cast<uint16_t*>(base);
     uint16_t* b_pad = reinterpret_cast<uint16_t*>(base + pad.bytes_a);
-    float* c_pad = reinterpret_cast<float*>(base + pad.bytes_a + pad.bytes_b);
-    float* inner_ws = reinterpret_cast<float*>(base + pad.bytes_a + pad.bytes_b + pad.bytes_c);
+    float* inner_ws = reinterpret_cast<float*>(base + pad.bytes_a + pad.bytes_b);
     e = pad_operands_launch(pad, b, m, k, n, static_cast<const uint16_t*>(A),
                             static_cast<const uint16_t*>(B), a_pad, b_pad, s, &launches);
     if (e == cudaSuccess)
       e = gemm_launch(st->info, pad_gemm, b, m, pad.k8, pad.n8,
                       pad.stage_a ? a_pad : static_cast<const uint16_t*>(A),
-                      pad.stage_b ? b_pad : static_cast<const uint16_t*>(B),
-                      pad.stage_c ? c_pad : C, pad_gemm.workspace_bytes ? inner_ws : nullptr, s,
-                      &launches, pad.stage_c ? true : overwrite);
-    if (e == cudaSuccess && pad.stage_c)
-      e = unpad_add_launch(pad, b, m, n, c_pad, C, overwrite, s, &launches);
+                      pad.stage_b ? b_pad : static_cast<const uint16_t*>(B), C,
+                      pad_gemm.workspace_bytes ? inner_ws : nullptr, s, &launches, overwrite, 0, nullptr,
+                      pad.stage_c ? n : 0);
   } else if (bt_fallback && b_layout != 1) {
     e = packed_fallback_launch(b_layout, b, m, k, n, static_cast<const uint16_t*>(A),
                                static_cast<const uint16_t*>(B), C, overwrite, s, &launches);
@@ -650,8 +647,8 @@ int morello_describe_route(int64_t b, int64_t m, int64_t k, int64_t n, char* tex
     const PadPlan pp = pad_plan(b, m, k, n, fake, fake, fake);
     kk = pp.k8;
     nn = pp.n8;
-    put("padded copies of%s%s%s to k=%lld n=%lld, then ", pp.stage_a ? " A" : "", pp.stage_b ? " B" : "",
-        pp.stage_c ? " C" : "", (long long)kk, (long long)nn);
+    put("padded copies of%s%s to k=%lld n=%lld%s, then ", pp.stage_a ? " A" : "", pp.stage_b ? " B" : "",
+        (long long)kk, (long long)nn, pp.stage_c ? " (C written from registers)" : "");
   }
   const int path = staged ? MORELLO_PATH_TCGEN05 : select_path(sms, b, m, k, n, fake, fake, fake);
   if (path == MORELLO_PATH_TCGEN05) {

@@ -22,6 +22,9 @@
 // MN-major operand, each 64-column group of the tile being one TMA box of 64 k rows.
 // Rows, columns and k blocks past the tensor edge are zero-filled by the TMA loads and
 // clipped by the TMA reduce, so m, n and k need not be multiples of the tile.
+// When the rows of C are not addressable by the TMA engine (a row pitch that is not a multiple
+// of 16 bytes, or a base that is not 16-byte aligned: the padded-copy route) the epilogue warps
+// add their sums to C straight from registers instead, one L2 reduction (or store) per element.
 // Every barrier wait is bounded (sm100::mbar_wait); on a timeout the block stops
 // issuing work, records a status word and exits after releasing its TMEM.
 #include <algorithm>
@@ -78,6 +81,7 @@ struct GemmParams {
   int64_t tiles;    // b * m_tiles * n_tiles
   int64_t whole;    // work items [0, whole) are whole tiles, in tile order;
   int64_t items;    // items [whole, items) are the column halves of tiles [whole, tiles)
+  int raster_g;     // rows of tiles per group of the tile order (see decode_item); 0: all of them
   int k_blocks;
   int ws_split;     // > 1: few tiles and a long k -- every tile's k range is cut into this many
                     // slices, each an item of its own whose sums go (as a plain store) to
@@ -92,6 +96,8 @@ struct GemmParams {
   int overwrite;   // 1: C = product (TMA store) instead of C += product (TMA reduce-add)
   int bt;          // 1: B is stored column-major, [b][n][k]: the K-major operand (boxes of 64 k x 64 columns)
   int a_box_rows;  // rows of A one TMA box brings: 128, or m rounded up to 16 when m < 128
+  int c_direct;    // 1: C is written from registers (its rows have c_cols columns, c_cols <= n,
+  int64_t c_cols;  //    and need no alignment beyond 4 bytes); the tensor map of C is not used
 };
 
 struct Barriers {
@@ -158,9 +164,23 @@ __device__ __forceinline__ Item decode_item(const GemmParams& p, int64_t t) {
     it.cols = kTileN / 2;
     it.n_off = (int)(h & 1) * (kTileN / 2);
   }
-  it.mt = (int)(tile % p.m_tiles);
-  it.nt = (int)((tile / p.m_tiles) % p.n_tiles);
-  it.bb = (int)(tile / ((int64_t)p.m_tiles * p.n_tiles));
+  // Tiles are numbered group by group: a group is raster_g rows of tiles (all of them when 0),
+  // walked row-fastest and then column by column, so that the tiles in flight at any time share
+  // a few rows of A and a few columns of B (both then stay in L2 while the wave passes).
+  // Batches are outermost.
+  const int64_t per_batch = (int64_t)p.m_tiles * p.n_tiles;
+  it.bb = (int)(tile / per_batch);
+  const int within = (int)(tile - it.bb * per_batch);
+  if (p.raster_g > 0) {
+    const int per_group = p.raster_g * p.n_tiles;
+    const int grp = within / per_group, r = within - grp * per_group;
+    const int rows = min(p.raster_g, p.m_tiles - grp * p.raster_g);
+    it.nt = r / rows;
+    it.mt = grp * p.raster_g + (r - it.nt * rows);
+  } else {
+    it.nt = within / p.m_tiles;
+    it.mt = within - it.nt * p.m_tiles;
+  }
   it.out_b = (int)(slice * p.bsz + it.bb);
   return it;
 }
@@ -199,7 +219,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     mbar_fence_init();
     tma_prefetch_descriptor(&map_a);
     tma_prefetch_descriptor(&map_b);
-    tma_prefetch_descriptor(&map_c);
+    if (!p.c_direct) tma_prefetch_descriptor(&map_c);
   }
   if (p.a_box_rows < kRowsPerCta) {
     // Few rows: the TMA box of A is only as high as m needs (a box that is mostly outside the
@@ -357,6 +377,48 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       const int col0 = it.nt * kTileN + it.n_off;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * kAccStride;
       const bool rows_live = row0 < p.m;   // warp-uniform
+      if (p.c_direct) {
+        // Straight from registers.  The 16-lane load shape hands every thread pairs of
+        // neighbouring columns of four rows, so that one warp-wide access covers 8 rows x 32
+        // contiguous bytes; every element goes out as one L2 reduction (or one store).
+        float* c_base = p.C + (int64_t)it.out_b * p.c_batch;
+        const int r_lo = row0 + (lane >> 2);            // this thread's rows: r_lo + 0, 8, 16, 24
+        const int c_lo = col0 + 2 * (lane & 3);
+#pragma unroll 1
+        for (int c = 0; c < it.cols; c += 64) {
+          uint32_t r0[32], r1[32];
+          tmem_ld_16x64(taddr + c, r0);                          // lanes 0-15 of the quarter
+          tmem_ld_16x64(taddr + ((uint32_t)16 << 16) + c, r1);   // lanes 16-31
+          tmem_ld_wait();
+          if (c + 64 >= it.cols) {
+            // The accumulator has left tensor memory: hand the buffer back to the MMA issuer.
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+              if constexpr (kPair) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->acc_empty[buf]), 0));
+              else mbar_arrive(&bars->acc_empty[buf]);
+            }
+          }
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+              const int row = r_lo + 8 * h;
+              if (row >= p.m) continue;
+#pragma unroll
+              for (int e = 0; e < 2; ++e) {
+                const int col = c_lo + c + 8 * q + e;
+                if (col >= p.c_cols) continue;
+                float* dst = c_base + (int64_t)row * p.c_cols + col;
+                const uint32_t v = (h < 2 ? r0 : r1)[4 * q + 2 * (h & 1) + e];
+                if (p.overwrite) *dst = __uint_as_float(v); else red_add_f32(dst, v);
+              }
+            }
+          }
+        }
+        if (++buf == 2) { buf = 0; acc_phase ^= 1; }
+        continue;
+      }
 #pragma unroll 1
       for (int c = 0; c < it.cols; c += kEpiCols) {
         const bool live = rows_live && (col0 + c < p.n);
@@ -456,7 +518,8 @@ struct SwapParams {
   int bt;           // 1: B is stored column-major, [b][n][k]
   int overwrite;    // 1: C = product instead of C += product
   int64_t m, n;
-  int64_t c_batch;  // m * n
+  int64_t c_batch;  // m * c_cols
+  int64_t c_cols;   // columns (and row pitch) of C: n, or fewer when B was padded with zero columns
   int k_blocks;
   int split_k;      // k slices per strip (cluster form: the slices of a strip are one cluster;
                     // otherwise every slice writes its own copy of the output, see the kernel)
@@ -640,7 +703,7 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
       const Work w = decode(t);
       const int slice = w.slice;
       const int64_t col = (int64_t)w.col0 + quarter * 32 + lane;   // this thread's column of C
-      const bool col_live = col < p.n;
+      const bool col_live = col < p.c_cols;
       // Without a cluster, slices > 1 means that C is partial[slice][b][m][n] in the workspace.
       const int64_t out_b = kClusterK ? w.bb : (int64_t)slice * p.bsz + w.bb;
       float* c_col = p.C + out_b * p.c_batch + col;
@@ -649,7 +712,7 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 #pragma unroll
       for (int i = 0; i < kRowsA; ++i) {
         const bool mine = !kClusterK || (i % p.split_k) == slice;
-        c_in[i] = (mine && col_live && i < p.m && !p.overwrite) ? c_col[(int64_t)i * p.n] : 0.f;
+        c_in[i] = (mine && col_live && i < p.m && !p.overwrite) ? c_col[(int64_t)i * p.c_cols] : 0.f;
       }
       if (ok) ok = mbar_wait(&bars->acc_full, acc_phase, abort_flag, p.status, 10);
       ok = __all_sync(0xffffffffu, ok);  // also reconverges the warp for the aligned TMEM loads
@@ -677,7 +740,7 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
               part[(g * 16 + i) * kSwapStripCols + quarter * 32 + lane] = __uint_as_float(r[i]);
             } else {
               if (col_live && g * 16 + i < p.m)
-                c_col[(int64_t)(g * 16 + i) * p.n] = c_in[g * 16 + i] + __uint_as_float(r[i]);
+                c_col[(int64_t)(g * 16 + i) * p.c_cols] = c_in[g * 16 + i] + __uint_as_float(r[i]);
             }
           }
         }
@@ -698,7 +761,7 @@ swap_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             const float* mine = part + i * kSwapStripCols + quarter * 32 + lane;
             float sum = *peer_shared(mine, 0u);
             for (int s2 = 1; s2 < p.split_k; ++s2) sum += *peer_shared(mine, (uint32_t)s2);
-            c_col[(int64_t)i * p.n] = c_in[i] + sum;
+            c_col[(int64_t)i * p.c_cols] = c_in[i] + sum;
           }
         }
         __syncwarp();
@@ -731,7 +794,8 @@ struct MapKey {
   const void* c;
   int64_t bsz, m, k, n;
   int bt;    // layout of B: 0 row-major, 1 column-major, >= 64 packed in strips of that many columns
-  int64_t c_bsz;   // batches of the output map: bsz, or slices x bsz when c is the workspace
+  int64_t c_bsz;   // batches of the output map: bsz, or slices x bsz when c is the workspace;
+                   // 0: no map of C is wanted (the kernel writes C from registers)
   bool operator==(const MapKey& o) const {
     return a == o.a && b == o.b && c == o.c && bsz == o.bsz && m == o.m && k == o.k && n == o.n &&
            bt == o.bt && c_bsz == o.c_bsz;
@@ -784,9 +848,10 @@ cudaError_t get_maps(const MapKey& key, CUtensorMap* ma, CUtensorMap* mb, CUtens
                              (uint64_t)key.k, (uint64_t)key.bsz, 64, kTileK,
                              CU_TENSOR_MAP_SWIZZLE_128B);
   if (err != cudaSuccess) return err;
-  err = make_tensor_map_3d(&e.map_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, key.c, (uint64_t)key.n,
-                           (uint64_t)key.m, (uint64_t)key.c_bsz, kEpiCols, 32,
-                           CU_TENSOR_MAP_SWIZZLE_128B);
+  if (key.c_bsz > 0)
+    err = make_tensor_map_3d(&e.map_c, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, key.c, (uint64_t)key.n,
+                             (uint64_t)key.m, (uint64_t)key.c_bsz, kEpiCols, 32,
+                             CU_TENSOR_MAP_SWIZZLE_128B);
   if (err != cudaSuccess) return err;
   e.stamp = ++g_stamp;
   e.valid = true;
@@ -881,6 +946,7 @@ int gemm_pair_units(int sms) { return pair_units(sms); }
 // block finished first.
 namespace {
 
+constexpr int kRasterRows = 8;                   // rows of tiles per group of the tile order
 constexpr int kWsMaxSplit = 8;
 constexpr int kWsMinBlocks = 16;                 // k blocks a slice keeps at least
 constexpr size_t kWsMaxBytes = size_t(64) << 20; // partial sums stay well inside L2
@@ -898,6 +964,7 @@ int ws_fit(int want, int64_t k_blocks, int64_t b, int64_t m, int64_t n) {
 
 GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob) {
   if (knob < 0) return GemmPlan{false, 0, 0, 0, false, 1, 1};
+  const int forced_g = (knob / 8192) % 64;
   const int forced_ws = (knob / 512) % 16;
   const bool halves = ((knob / 256) % 2) == 0;
   knob %= 256;
@@ -909,6 +976,9 @@ GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob
       plan.workspace_bytes = (size_t)plan.ws_split * b * m * n * 4;
       plan.halves = false;
     }
+    // The tile order: groups of kRasterRows rows of tiles unless the knob says otherwise (63: a
+    // column of tiles at a time).
+    plan.raster_g = forced_g == 63 ? 0 : forced_g != 0 ? forced_g : kRasterRows;
     return plan;
   };
   // By shape, the k slices of `tiles` items on `units` units.
@@ -995,8 +1065,8 @@ namespace {
 template <bool kPair, int kTileN>
 cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, int64_t n,
                         const CUtensorMap& map_a, const CUtensorMap& map_b,
-                        const CUtensorMap& map_c, float* C, bool halves, int ws_split,
-                        bool overwrite, int bt, const KSegments* seg, cudaStream_t stream) {
+                        const CUtensorMap& map_c, float* C, bool halves, int ws_split, int raster_g,
+                        int64_t c_cols, bool overwrite, int bt, const KSegments* seg, cudaStream_t stream) {
   using S = Shape<kPair, kTileN>;
   const cudaError_t attr_err = set_smem_attribute<kPair, kTileN>();
   if (attr_err != cudaSuccess) return attr_err;
@@ -1004,7 +1074,9 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   GemmParams p{};
   p.C = C;
   p.m = m; p.n = n; p.k = k;
-  p.c_batch = m * n;
+  p.c_direct = c_cols > 0 ? 1 : 0;
+  p.c_cols = c_cols > 0 ? c_cols : n;
+  p.c_batch = m * p.c_cols;
   p.m_tiles = (int)((m + S::kTileM - 1) / S::kTileM);
   p.n_tiles = (int)((n + kTileN - 1) / kTileN);
   p.tiles = b * p.m_tiles * (int64_t)p.n_tiles;
@@ -1018,6 +1090,7 @@ cudaError_t launch_gemm(const DeviceInfo& dev, int64_t b, int64_t m, int64_t k, 
   p.pack_strip = bt >= 64 ? bt : 0;
   p.pack_strips = bt >= 64 ? (int)((n + bt - 1) / bt) : 0;
   p.bsz = b;
+  p.raster_g = raster_g > 0 && raster_g < p.m_tiles ? raster_g : 0;
   if (seg) { p.seg_blocks = seg->blocks; p.seg_a = seg->a_terms; p.seg_b = seg->b_terms; }
   p.ws_split = std::max(1, ws_split);
   p.kb_per_slice = (p.k_blocks + p.ws_split - 1) / p.ws_split;
@@ -1070,7 +1143,7 @@ int64_t swap_resident(int sms) { return (int64_t)sms * (kRowsA <= 16 ? 2 : 1); }
 
 template <int kRowsA, bool kClusterK, bool kPersistent>
 cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_t m, int64_t k, int64_t n,
-                             const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
+                             const CUtensorMap& map_a, const CUtensorMap& map_b, float* C, int64_t c_cols,
                              bool overwrite, int bt, const KSegments* seg, cudaStream_t stream) {
   using S = SwapShape<kRowsA>;
   static PerDeviceOnce once;   // the attribute belongs to the current device's copy of the kernel
@@ -1085,7 +1158,8 @@ cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_
   p.pack_strips = bt >= 64 ? (int)((n + bt - 1) / bt) : 0;
   p.overwrite = overwrite ? 1 : 0;
   p.m = m; p.n = n;
-  p.c_batch = m * n;
+  p.c_cols = c_cols > 0 ? c_cols : n;
+  p.c_batch = m * p.c_cols;
   p.k_blocks = (int)((k + kTileK - 1) / kTileK);
   p.split_k = std::max(1, split);
   p.bsz = b;
@@ -1133,17 +1207,17 @@ cudaError_t launch_swap_form(const DeviceInfo& dev, int split, int64_t b, int64_
 template <int kRowsA>
 cudaError_t launch_swap(const DeviceInfo& dev, int split, int ws_split, int64_t b, int64_t m, int64_t k,
                         int64_t n, const CUtensorMap& map_a, const CUtensorMap& map_b, float* C,
-                        bool overwrite, int bt, const KSegments* seg, cudaStream_t stream) {
+                        int64_t c_cols, bool overwrite, int bt, const KSegments* seg, cudaStream_t stream) {
   if (split > 1)
-    return launch_swap_form<kRowsA, true, false>(dev, split, b, m, k, n, map_a, map_b, C, overwrite, bt, seg,
-                                                 stream);
+    return launch_swap_form<kRowsA, true, false>(dev, split, b, m, k, n, map_a, map_b, C, c_cols, overwrite, bt,
+                                                 seg, stream);
   // More items than blocks fit at once (and batches beyond a grid dimension): persistent.
   const int64_t items = b * ((n + kSwapStripCols - 1) / kSwapStripCols) * std::max(1, ws_split);
   if (items > swap_resident<kRowsA>(dev.sms) || b > 65535)
-    return launch_swap_form<kRowsA, false, true>(dev, ws_split, b, m, k, n, map_a, map_b, C, overwrite, bt,
-                                                 seg, stream);
-  return launch_swap_form<kRowsA, false, false>(dev, ws_split, b, m, k, n, map_a, map_b, C, overwrite, bt,
-                                                seg, stream);
+    return launch_swap_form<kRowsA, false, true>(dev, ws_split, b, m, k, n, map_a, map_b, C, c_cols, overwrite,
+                                                 bt, seg, stream);
+  return launch_swap_form<kRowsA, false, false>(dev, ws_split, b, m, k, n, map_a, map_b, C, c_cols, overwrite,
+                                                bt, seg, stream);
 }
 
 }  // namespace
@@ -1151,38 +1225,45 @@ cudaError_t launch_swap(const DeviceInfo& dev, int split, int ws_split, int64_t 
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m, int64_t k,
                         int64_t n, const uint16_t* A, const uint16_t* B, float* C, float* workspace,
                         cudaStream_t stream, uint64_t* launches, bool overwrite, int bt,
-                        const KSegments* seg) {
+                        const KSegments* seg, int64_t c_cols) {
   // With k slices through the workspace the kernels write partial[slice][b][m][n] there (plain
   // stores) and the reduce launch below adds the slices and C.
   const bool sliced = plan.ws_split > 1;
   if (sliced && !workspace) return cudaErrorInvalidValue;
+  if (c_cols < 0 || c_cols > n) return cudaErrorInvalidValue;
   float* out = sliced ? workspace : C;
   const bool out_overwrite = sliced ? true : overwrite;
+  // c_cols > 0: C is [b][m][c_cols], written from registers by the kernels (or, sliced, by the
+  // reduce launch); the partial sums in the workspace keep the kernels' own n columns.
+  const int64_t direct = sliced ? 0 : c_cols;
   CUtensorMap map_a, map_b, map_c;
   // With segments the stored operands are shorter along k than the call's k range.
   if (seg && (seg->blocks <= 0 || k % (64ll * seg->blocks) != 0 || k / (64ll * seg->blocks) > 8))
     return cudaErrorInvalidValue;
-  cudaError_t e = get_maps(MapKey{A, B, out, b, m, seg ? seg->k_stored : k, n, bt, sliced ? plan.ws_split * b : b},
+  cudaError_t e = get_maps(MapKey{A, B, out, b, m, seg ? seg->k_stored : k, n, bt,
+                                  direct > 0 ? 0 : sliced ? plan.ws_split * b : b},
                            &map_a, &map_b, &map_c);
   if (e != cudaSuccess) return e;
   const int code = plan.form * 1000 + plan.tile_n;
-  const int wss = plan.ws_split;
+  const int wss = plan.ws_split, rg = plan.raster_g;
+  const bool hv = plan.halves;
   switch (code) {
-    case 3016: e = launch_swap<16>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, seg, stream); break;
-    case 3032: e = launch_swap<32>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, seg, stream); break;
-    case 3048: e = launch_swap<48>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, seg, stream); break;
-    case 3064: e = launch_swap<64>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, out_overwrite, bt, seg, stream); break;
-    case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, seg, stream); break;
-    case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, seg, stream); break;
-    case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, seg, stream); break;
-    case 2128: e = launch_gemm<true, 128>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, seg, stream); break;
-    case 2256: e = launch_gemm<true, 256>(dev, b, m, k, n, map_a, map_b, map_c, out, plan.halves, wss, out_overwrite, bt, seg, stream); break;
+    case 3016: e = launch_swap<16>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, direct, out_overwrite, bt, seg, stream); break;
+    case 3032: e = launch_swap<32>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, direct, out_overwrite, bt, seg, stream); break;
+    case 3048: e = launch_swap<48>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, direct, out_overwrite, bt, seg, stream); break;
+    case 3064: e = launch_swap<64>(dev, plan.split_k, wss, b, m, k, n, map_a, map_b, out, direct, out_overwrite, bt, seg, stream); break;
+    case 1064: e = launch_gemm<false, 64>(dev, b, m, k, n, map_a, map_b, map_c, out, hv, wss, rg, direct, out_overwrite, bt, seg, stream); break;
+    case 1128: e = launch_gemm<false, 128>(dev, b, m, k, n, map_a, map_b, map_c, out, hv, wss, rg, direct, out_overwrite, bt, seg, stream); break;
+    case 1256: e = launch_gemm<false, 256>(dev, b, m, k, n, map_a, map_b, map_c, out, hv, wss, rg, direct, out_overwrite, bt, seg, stream); break;
+    case 2128: e = launch_gemm<true, 128>(dev, b, m, k, n, map_a, map_b, map_c, out, hv, wss, rg, direct, out_overwrite, bt, seg, stream); break;
+    case 2256: e = launch_gemm<true, 256>(dev, b, m, k, n, map_a, map_b, map_c, out, hv, wss, rg, direct, out_overwrite, bt, seg, stream); break;
     default: return cudaErrorInvalidValue;
   }
   if (e != cudaSuccess) return e;
   ++*launches;
   if (sliced) {
-    e = skinny_reduce_launch(workspace, C, b, (int)m, n, m * n, plan.ws_split, stream, overwrite);
+    e = skinny_reduce_launch(workspace, C, b, (int)m, n, m * (c_cols > 0 ? c_cols : n), plan.ws_split, stream,
+                             overwrite, c_cols);
     if (e != cudaSuccess) return e;
     ++*launches;
   }

@@ -83,9 +83,11 @@ cudaError_t skinny_launch(const SkinnyPlan& plan, int64_t b, int m, int64_t k, i
 
 // Enqueues the slice-ordered reduce: C[b, i, :] += partial[0] + partial[1] + ... for the
 // b * m * n sums of one row chunk (partial is [split_k][b][m][n], c_batch the batch stride of C).
+// c_cols > 0: C is dense [b][m][c_cols] with c_cols <= n; the columns of the partial sums past
+// c_cols (sums over zero padding) are dropped.
 cudaError_t skinny_reduce_launch(const float* partial, float* C, int64_t b, int m, int64_t n,
                                  int64_t c_batch, int split_k, cudaStream_t stream,
-                                 bool overwrite = false);
+                                 bool overwrite = false, int64_t c_cols = 0);
 
 // ---- streaming GEMV (FP32 FMA, B through a TMA ring, m <= 4) ------------------
 struct StreamPlan {
@@ -119,8 +121,10 @@ cudaError_t f32_split_launch(int64_t b, int64_t m, int64_t k, int64_t n, const f
 // ---- zero-padded copies of operands the TMA engine cannot address --------------
 struct PadPlan {
   int64_t k8, n8;                    // k and n rounded up to multiples of 8
-  bool stage_a, stage_b, stage_c;    // which operands go through a padded copy
-  size_t bytes_a, bytes_b, bytes_c;  // their sizes in the workspace (multiples of 256)
+  bool stage_a, stage_b;             // which operands go through a padded copy
+  bool stage_c;                      // C's rows are not TMA-addressable: the kernels write them
+                                     // from registers (no copy of C is made)
+  size_t bytes_a, bytes_b;           // sizes of the copies in the workspace (multiples of 256)
 };
 // Which operands need a copy for these extents and pointers.
 PadPlan pad_plan(int64_t b, int64_t m, int64_t k, int64_t n, const void* A, const void* B,
@@ -128,9 +132,6 @@ PadPlan pad_plan(int64_t b, int64_t m, int64_t k, int64_t n, const void* A, cons
 cudaError_t pad_operands_launch(const PadPlan& p, int64_t b, int64_t m, int64_t k, int64_t n,
                                 const uint16_t* A, const uint16_t* B, uint16_t* A_pad,
                                 uint16_t* B_pad, cudaStream_t stream, uint64_t* launches);
-// C (+)= the first n columns of C_pad[b][m][n8].
-cudaError_t unpad_add_launch(const PadPlan& p, int64_t b, int64_t m, int64_t n, const float* C_pad,
-                             float* C, bool overwrite, cudaStream_t stream, uint64_t* launches);
 
 // ---- tcgen05 path ------------------------------------------------------------
 struct GemmPlan {
@@ -142,13 +143,15 @@ struct GemmPlan {
   int split_k;   // operand-swapped kernel only: k slices per strip, added inside a cluster (1, 2, 4, 8)
   int ws_split;  // > 1: k slices whose sums go to partial[slice][b][m][n] in the workspace and are
                  // added, slice by slice and then to C, by the reduce kernel
+  int raster_g = 0;  // rows of tiles per group of the tile order; 0: a column of tiles at a time
 };
 
 bool gemm_shape_supported(int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
                           const void* B, const void* C);
 // `knob`: 0 = by shape; otherwise form + 16 * (tile columns / 64) [+ 256 to keep the last wave's
-// tiles whole], the first two parts 0 = by shape; with form 3 the second part is the number of k
-// slices (0 = by shape, 1, 2, 4 or 8).
+// tiles whole] [+ 512 * k slices through the workspace] [+ 8192 * rows of tiles per group of the
+// tile order, 63 = a column of tiles at a time], every part 0 = by shape; with form 3 the second
+// part is the number of k slices added inside a cluster (0 = by shape, 1, 2, 4 or 8).
 GemmPlan gemm_plan(int sms, int64_t b, int64_t m, int64_t k, int64_t n, int knob);
 // The k range as a sequence of up to 8 equal segments, each reading one of the stored k ranges
 // of A and of B (float32 inputs: six products of three stored terms each, see f32_split.cu):
@@ -163,10 +166,14 @@ struct KSegments {
 int gemm_pair_units(int sms);
 // b_layout: 0 = B row-major [b][k][n], 1 = column-major [b][n][k], a multiple of 64 = packed in
 // strips of that many columns, [b][ceil(n / strip)][k][strip].
+// c_cols: 0 = C is [b][m][n] and 16-byte aligned (addressed by the TMA engine); otherwise C is
+// [b][m][c_cols] with c_cols <= n (B carries n - c_cols columns of zero padding) and any 4-byte
+// alignment, and is written from registers, element by element.
 cudaError_t gemm_launch(const DeviceInfo& dev, const GemmPlan& plan, int64_t b, int64_t m,
                         int64_t k, int64_t n, const uint16_t* A, const uint16_t* B, float* C,
                         float* workspace, cudaStream_t stream, uint64_t* launches,
-                        bool overwrite = false, int b_layout = 0, const KSegments* seg = nullptr);
+                        bool overwrite = false, int b_layout = 0, const KSegments* seg = nullptr,
+                        int64_t c_cols = 0);
 
 // ---- B stored column-major where the TMA engine cannot address it ------------
 // C[b, i, j] (+)= sum_p A[b, i, p] * Bt[b, j, p]: one warp per output column, lanes stride over

@@ -3,21 +3,22 @@
 // zero-padded, 16-byte-aligned buffers in the workspace,
 //     A'[b][m][k8]  (k8 = k rounded up to 8; the added columns are zero),
 //     B'[b][k8][n8] (n8 = n rounded up to 8; the added rows and columns are zero),
-// the tensor-core kernels compute MatmulAccum(b, m, k8, n8) on them -- the zero padding adds
-// exact zeros to every sum -- and, when C's rows cannot be addressed either, the product goes
-// to C'[b][m][n8] first and one elementwise launch adds (or, for Matmul, copies) its first n
-// columns to C.  C is still added exactly once, last, to the complete sum.
+// by one launch, and the tensor-core kernels compute MatmulAccum(b, m, k8, n8) on them -- the
+// zero padding adds exact zeros to every sum.  When C's rows cannot be addressed by the TMA
+// engine either (n % 8 != 0 or a base that is not 16-byte aligned) the kernels' epilogues add
+// their sums to the first n columns of each row of C straight from registers; C is still added
+// exactly once, last, to the complete sum.
 #include "internal.h"
 #include "sm100.cuh"
 
 namespace morello {
 namespace {
 
-// The copies, the tensor-core call and the unpad-add form a chain of short launches: each is
-// launched with programmatic stream serialisation, waits for its predecessor before it touches
-// global memory and lets its successor's blocks be scheduled right away, so that the launch
-// latencies overlap.  (Every kernel of the chain executes the wait, so "the predecessor has
-// completed" carries through the whole chain.)
+// The copy launch and the tensor-core call form a chain of short launches: each is launched
+// with programmatic stream serialisation, waits for its predecessor before it touches global
+// memory and lets its successor's blocks be scheduled right away, so that the launch latencies
+// overlap.  (Every kernel of the chain executes the wait, so "the predecessor has completed"
+// carries through the whole chain.)
 template <typename... KArgs, typename... Args>
 cudaError_t launch_chained(void (*kern)(KArgs...), unsigned blocks, cudaStream_t stream, Args... args) {
   cudaLaunchConfig_t cfg{};
@@ -35,25 +36,27 @@ cudaError_t launch_chained(void (*kern)(KArgs...), unsigned blocks, cudaStream_t
 
 // dst[bb][r][c] = src[bb][r][c] inside the source extents, else 0; dst is [b][rows_out][cols_out]
 // with cols_out % 8 == 0 and a 16-byte-aligned base.  One thread per 8 output elements.
-__global__ void __launch_bounds__(256)
-pad_bf16_kernel(const uint16_t* __restrict__ src, uint4* __restrict__ dst, int64_t b, int64_t rows_in,
-                int64_t cols_in, int64_t rows_out, int64_t cols_out) {
-  const int64_t groups = cols_out / 8;
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  sm100::pdl_wait();
-  sm100::pdl_release();
-  if (idx >= b * rows_out * groups) return;
+struct PadJob {
+  const uint16_t* src;
+  uint4* dst;
+  int64_t rows_in, cols_in, rows_out, cols_out;
+  int64_t threads;   // b * rows_out * cols_out / 8; 0: nothing to copy
+};
+
+__device__ __forceinline__ void pad_one(const PadJob& j, int64_t idx) {
+  const int64_t groups = j.cols_out / 8;
   const int64_t g = idx % groups;
-  const int64_t r = (idx / groups) % rows_out;
-  const int64_t bb = idx / (groups * rows_out);
+  const int64_t r = (idx / groups) % j.rows_out;
+  const int64_t bb = idx / (groups * j.rows_out);
   uint32_t w[4] = {0u, 0u, 0u, 0u};
-  if (r < rows_in) {
-    const uint16_t* row = src + (bb * rows_in + r) * cols_in;
+  if (r < j.rows_in) {
+    const uint16_t* row = j.src + (bb * j.rows_in + r) * j.cols_in;
     const int64_t c0 = g * 8;
     const uint16_t* at = row + c0;
-    if (c0 + 8 <= cols_in) {
+    if (c0 + 8 <= j.cols_in) {
       // Eight elements inside the row: 32-bit loads where the address allows (the source rows
-      // are only 2-byte aligned), 4 or 5 loads instead of 8.
+      // are only 2-byte aligned), 4 or 5 loads instead of 8.  (Two aligned 16-byte granules and
+      // a funnel shift instead were measured slower.)
       if ((reinterpret_cast<uintptr_t>(at) & 2u) == 0) {
         const uint32_t* q = reinterpret_cast<const uint32_t*>(at);
         w[0] = q[0]; w[1] = q[1]; w[2] = q[2]; w[3] = q[3];
@@ -69,25 +72,22 @@ pad_bf16_kernel(const uint16_t* __restrict__ src, uint4* __restrict__ dst, int64
     } else {
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
-        const uint32_t v = (c0 + e < cols_in) ? (uint32_t)at[e] : 0u;
+        const uint32_t v = (c0 + e < j.cols_in) ? (uint32_t)at[e] : 0u;
         w[e >> 1] |= v << ((e & 1) * 16);
       }
     }
   }
-  dst[idx] = make_uint4(w[0], w[1], w[2], w[3]);
+  j.dst[idx] = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// C[bb][i][j] = (overwrite ? 0 : C[bb][i][j]) + P[bb][i][j] for j < n; P is [b][m][n8].
+// Both copies in one launch: threads [0, a.threads) pad A, the next b.threads pad B.
 __global__ void __launch_bounds__(256)
-unpad_add_kernel(const float* __restrict__ P, float* __restrict__ C, int64_t rows, int64_t n,
-                 int64_t n8, int overwrite) {
+pad_operands_kernel(const PadJob a, const PadJob b) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   sm100::pdl_wait();
   sm100::pdl_release();
-  if (idx >= rows * n) return;
-  const int64_t r = idx / n, j = idx - r * n;
-  const float sum = P[r * n8 + j];
-  C[idx] = overwrite ? sum : C[idx] + sum;
+  if (idx < a.threads) pad_one(a, idx);
+  else if (idx - a.threads < b.threads) pad_one(b, idx - a.threads);
 }
 
 size_t round256(size_t x) { return (x + 255) / 256 * 256; }
@@ -105,35 +105,20 @@ PadPlan pad_plan(int64_t b, int64_t m, int64_t k, int64_t n, const void* A, cons
   p.stage_c = n_odd || reinterpret_cast<uintptr_t>(C) % 16 != 0;
   p.bytes_a = p.stage_a ? round256((size_t)b * m * p.k8 * 2) : 0;
   p.bytes_b = p.stage_b ? round256((size_t)b * p.k8 * p.n8 * 2) : 0;
-  p.bytes_c = p.stage_c ? round256((size_t)b * m * p.n8 * 4) : 0;
   return p;
 }
 
 cudaError_t pad_operands_launch(const PadPlan& p, int64_t b, int64_t m, int64_t k, int64_t n,
                                 const uint16_t* A, const uint16_t* B, uint16_t* A_pad,
                                 uint16_t* B_pad, cudaStream_t stream, uint64_t* launches) {
-  if (p.stage_a) {
-    const int64_t threads = b * m * (p.k8 / 8);
-    const cudaError_t e = launch_chained(pad_bf16_kernel, (unsigned)((threads + 255) / 256), stream, A,
-                                         reinterpret_cast<uint4*>(A_pad), b, m, k, m, p.k8);
-    if (e != cudaSuccess) return e;
-    ++*launches;
-  }
-  if (p.stage_b) {
-    const int64_t threads = b * p.k8 * (p.n8 / 8);
-    const cudaError_t e = launch_chained(pad_bf16_kernel, (unsigned)((threads + 255) / 256), stream, B,
-                                         reinterpret_cast<uint4*>(B_pad), b, k, n, p.k8, p.n8);
-    if (e != cudaSuccess) return e;
-    ++*launches;
-  }
-  return cudaSuccess;
-}
-
-cudaError_t unpad_add_launch(const PadPlan& p, int64_t b, int64_t m, int64_t n, const float* C_pad,
-                             float* C, bool overwrite, cudaStream_t stream, uint64_t* launches) {
-  const int64_t total = b * m * n;
-  const cudaError_t e = launch_chained(unpad_add_kernel, (unsigned)((total + 255) / 256), stream, C_pad, C,
-                                       b * m, n, p.n8, overwrite ? 1 : 0);
+  PadJob ja{}, jb{};
+  if (p.stage_a) ja = PadJob{A, reinterpret_cast<uint4*>(A_pad), m, k, m, p.k8, b * m * (p.k8 / 8)};
+  if (p.stage_b) jb = PadJob{B, reinterpret_cast<uint4*>(B_pad), k, n, p.k8, p.n8, b * p.k8 * (p.n8 / 8)};
+  const int64_t threads = ja.threads + jb.threads;
+  if (threads == 0) return cudaSuccess;
+  const int64_t blocks = (threads + 255) / 256;
+  if (blocks >= (1ll << 31)) return cudaErrorInvalidValue;
+  const cudaError_t e = launch_chained(pad_operands_kernel, (unsigned)blocks, stream, ja, jb);
   if (e != cudaSuccess) return e;
   ++*launches;
   return cudaSuccess;

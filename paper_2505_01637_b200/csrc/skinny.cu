@@ -308,6 +308,22 @@ reduce4_kernel(const float4* __restrict__ partial, float* __restrict__ C, int64_
   *c = sum;
 }
 
+// The same sums when C has fewer columns than the partial sums (zero-padded operands): C is dense
+// [rows][c_cols], the partial sums are [split_k][rows][n]; one thread per element of C.
+__global__ void __launch_bounds__(256)
+reduce_narrow_kernel(const float* __restrict__ partial, float* __restrict__ C, int64_t rows, int64_t n,
+                     int64_t c_cols, int split_k, int overwrite) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  pdl_wait();
+  pdl_release();
+  if (idx >= rows * c_cols) return;
+  const int64_t r = idx / c_cols, j = idx - r * c_cols;
+  const float* src = partial + r * n + j;
+  float sum = src[0];
+  for (int s = 1; s < split_k; ++s) sum += src[(int64_t)s * rows * n];
+  C[idx] = overwrite ? sum : C[idx] + sum;
+}
+
 // Launch with programmatic stream serialisation (see pdl_wait above).
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, int threads, size_t smem,
@@ -576,7 +592,13 @@ cudaError_t packed_fallback_launch(int64_t strip, int64_t b, int64_t m, int64_t 
 }
 
 cudaError_t skinny_reduce_launch(const float* partial, float* C, int64_t b, int m, int64_t n,
-                                 int64_t c_batch, int split_k, cudaStream_t stream, bool overwrite) {
+                                 int64_t c_batch, int split_k, cudaStream_t stream, bool overwrite,
+                                 int64_t c_cols) {
+  if (c_cols > 0 && c_cols != n) {
+    const int64_t rows = b * m, blocks = (rows * c_cols + 255) / 256;
+    return launch_pdl(reduce_narrow_kernel, dim3((unsigned)blocks, 1, 1), 256, 0, stream, partial, C, rows, n,
+                      c_cols, split_k, overwrite ? 1 : 0);
+  }
   const int64_t total = b * m * n;
   const int64_t mn = (int64_t)m * n;
   if (mn % 4 == 0 && c_batch % 4 == 0 && reinterpret_cast<uintptr_t>(partial) % 16 == 0 &&

@@ -70,7 +70,8 @@ def test_selector_is_shape_based(mb):
     assert mb.morello_select_path(1, 2, 2048, 1024) == mb.MORELLO_PATH_TCGEN05     # few columns: k is cut instead
     assert mb.morello_select_path(1, 16, 4096, 64) == mb.MORELLO_PATH_TCGEN05
     assert mb.morello_select_path(1, 8, 4096, 60) == mb.MORELLO_PATH_SKINNY         # n % 8 != 0: TMA cannot address it
-    assert mb.morello_select_path(1, 17, 100, 100) == mb.MORELLO_PATH_SKINNY       # ... and too small to be worth copying
+    assert mb.morello_select_path(1, 16, 100, 100) == mb.MORELLO_PATH_SKINNY       # ... one chunk of rows: not worth copying
+    assert mb.morello_select_path(1, 17, 100, 100) == mb.MORELLO_PATH_TCGEN05      # ... two chunks: padded copies are cheaper
     assert mb.morello_select_path(1, 4096, 4096, 4095) == mb.MORELLO_PATH_TCGEN05  # ... through zero-padded copies
     assert mb.morello_select_path(1, 512, 1001, 1000) == mb.MORELLO_PATH_TCGEN05   # k % 8 != 0 likewise
     assert mb.morello_select_path(1, 4096, 4096, 4096) == mb.MORELLO_PATH_TCGEN05
@@ -89,7 +90,8 @@ def test_route_description_names_the_kernel(mb):
     assert "one CTA per 128 x" in d(1, 128, 2048, 16384)
     assert "k slices through the workspace" in d(1, 512, 16384, 2048)
     assert "added inside a cluster" in d(1, 16, 16384, 2048)
-    assert d(1, 2048, 2047, 2049).startswith("padded copies of A B C to k=2048 n=2056, then tcgen05")
+    assert d(1, 2048, 2047, 2049).startswith("padded copies of A B to k=2048 n=2056 (C written from registers), then tcgen05")
+    assert d(1, 512, 1001, 1000).startswith("padded copies of A B to k=1008 n=1000, then tcgen05")
     assert d(1, 4, 4, 16).startswith("fma skinny_kernel")
     assert "shifted columns" in d(1, 1, 2048, 16383)
     assert d(0, 4, 4, 4).startswith("nothing to launch")

@@ -27,9 +27,12 @@ TC = mb.MORELLO_PATH_TCGEN05
     (3, 64, 64, 64),
     (1, 1024, 128, 2048),   # more tiles than fit one wave of a small grid
 ])
-@pytest.mark.parametrize("form", [1, 2, 16 + 1, 32 + 1, 32 + 2, 64 + 1, 64 + 2])
+@pytest.mark.parametrize("form", [1, 2, 16 + 1, 32 + 1, 32 + 2, 64 + 1, 64 + 2,
+                                  64 + 2 + 8192 * 1, 32 + 1 + 8192 * 3, 16 + 1 + 8192 * 63])
 def test_integer_inputs_bit_exact(shape, form):
-    # form % 16: one CTA per tile / a CTA pair per tile; form // 16: tile columns / 64 (0 = by shape)
+    # form % 16: one CTA per tile / a CTA pair per tile; (form // 16) % 16: tile columns / 64 (0 = by
+    # shape); form // 8192: rows of tiles per group of the tile order (0 = by shape, 63 = a column
+    # of tiles at a time)
     b, m, k, n = shape
     A, B, C = w.make(b, m, k, n, seed=sum(shape), ab="int4", c="normal")
     check_full(A, B, C, integer=True, path=TC, split_k=form, what="tcgen05 form %d %s" % (form, shape))
