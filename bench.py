@@ -12,11 +12,16 @@ buffers so that no call finds its input in L2.
 
 How the headline is timed: every rotating buffer set is called once (untimed,
 so that no first-use cost of a buffer lands in the timed region), then W
-warm-up steps, then the K-step loop runs R times back to back on the stream
-(R >= 25 and at least 50 ms of work), each loop bracketed by its own pair of
-CUDA events, the whole region by a barrier + synchronize on both sides.
-`ms_per_step` is the MEDIAN loop divided by K; the minimum, maximum and mean
-are printed beside it, and `clocks` describes exactly that region.
+warm-up steps, then the K-step loop runs back to back on the stream, in R
+blocks (R >= 25 and at least 50 ms of work) of J loops each (J * K >= 200
+steps), every block bracketed by its own pair of CUDA events, the whole region
+by a barrier + synchronize on both sides.  An event between two launches keeps
+the second from overlapping the first's tail (calls are chained by programmatic
+dependent launch), which back-to-back calls of a user do not suffer: hence
+blocks of at least 200 steps per event pair.  `ms_per_step` is the MEDIAN
+block divided by its steps; the minimum, maximum and mean are printed beside
+it, `timing.single_loop_us_per_step` is one K-step loop alone between two
+synchronisations, and `clocks` describes exactly the timed region.
 
 `e2e` is the same metric through the host-buffer entry point, host<->device
 copies inside the timed region.  `configs` reports the other shapes (GEMM ones
@@ -56,9 +61,10 @@ TARGET_TENSOR_FRAC_OF_NOMINAL = 0.70    # the large GEMMs: >= 70 % of the dense 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 HEADLINE = 1            # index into workloads.CONFIGS: the 1 x 2048 x 16384 GEMV
 ROTATE = 8              # distinct B buffers: 8 x 64 MiB = 512 MiB > 4 x the 126 MB L2
-MIN_LOOPS = 25          # the K-step loop is repeated at least this often ...
+MIN_LOOPS = 25          # event-bracketed blocks of K-step loops: at least this many ...
 MIN_TIMED_SECONDS = 0.05    # ... and until this much work has been timed
 MAX_LOOPS = 4000
+MIN_BLOCK_STEPS = 200   # steps per event pair: an event between launches costs the next its overlap
 
 
 def workload_name(cfg):
@@ -290,10 +296,15 @@ def whole_job_value(units_per_rank_per_step, steps, world, seconds):
 
 
 def loop_count(pilot_seconds):
-    """How often the K-step loop is repeated, from the time of one pilot loop."""
+    """How many event-bracketed blocks are timed, from the time of one pilot block."""
     if pilot_seconds <= 0:
         return MIN_LOOPS
     return int(min(MAX_LOOPS, max(MIN_LOOPS, math.ceil(MIN_TIMED_SECONDS / pilot_seconds))))
+
+
+def loops_per_block(steps):
+    """K-step loops per event pair, so that a block has at least MIN_BLOCK_STEPS steps."""
+    return max(1, -(-MIN_BLOCK_STEPS // steps))
 
 
 def spread(loops, steps):
@@ -572,28 +583,32 @@ def run_ours(args):
     torch.cuda.synchronize()
     for i in range(args.warmup):
         step(i)
-    pilot = max_over_ranks(time_calls(torch, step, args.steps, 0), dist, "cuda")   # one more untimed loop
-    loops_n = loop_count(pilot)
+    single = max_over_ranks(time_calls(torch, step, args.steps, 0), dist, "cuda")   # one K-step loop alone
+    block_steps = loops_per_block(args.steps) * args.steps
+    loops_n = loop_count(single * block_steps / args.steps)
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
         torch.cuda.synchronize()
     l0 = mb.morello_launch_count()
     t0 = time.perf_counter()
-    loops = timed_loops(torch, step, args.steps, loops_n)     # ends with a synchronize
+    loops = timed_loops(torch, step, block_steps, loops_n)    # ends with a synchronize
     headline_window = [(t0, time.perf_counter())]
     if dist is not None:
         dist.barrier()
         torch.cuda.synchronize()
     launches = mb.morello_launch_count() - l0
-    sec = max_over_ranks(statistics.median(loops), dist, "cuda")      # the median K-step loop
+    # the median block, scaled to the K steps of one loop
+    sec = max_over_ranks(statistics.median(loops), dist, "cuda") * args.steps / block_steps
     st, detail = mb.morello_read_device_status()
     if st != 0:
         raise RuntimeError("device status %d (0x%x)" % (st, detail))
     value = whole_job_value(cfg.algorithmic_bytes, args.steps, world, sec) / 1e9
-    timing = spread(loops, args.steps)
-    timing["loop_us"] = [round(x * 1e6, 2) for x in loops]
-    timing["whole_region_us_per_step"] = sum(loops) / (len(loops) * args.steps) * 1e6
+    timing = spread(loops, block_steps)
+    timing["steps_per_block"] = block_steps
+    timing["block_us"] = [round(x * 1e6, 2) for x in loops]
+    timing["whole_region_us_per_step"] = sum(loops) / (len(loops) * block_steps) * 1e6
+    timing["single_loop_us_per_step"] = single / args.steps * 1e6
 
     # ---- the same calls on ONE set of buffers (how the config is worded: "timed warm over 1000
     # calls"); B's 64 MiB fit the 126 MB L2, so this figure is L2-assisted and is not the headline
@@ -697,7 +712,8 @@ def run_ours(args):
                 ("mid_128x2048x16384", (1, 128, 2048, 16384), 200, "128 rows on a streaming shape"),
                 ("mid_256x4096x4096", (1, 256, 4096, 4096), 200, "few tiles, k slices"),
                 ("mid_512x4096x4096", (1, 512, 4096, 4096), 200, "few tiles"),
-                ("mid_256x8192x8192", (1, 256, 8192, 8192), 100, "one row of pair tiles, long k")):
+                ("mid_256x8192x8192", (1, 256, 8192, 8192), 100, "one row of pair tiles, long k"),
+                ("gemm_8192_cube", (1, 8192, 8192, 8192), 6, "32 x 32 pair tiles: the tile order's groups of 8 rows keep A and B in L2")):
             extra.append(bench_shape(torch, mb, name, shape, iters, peaks, windows, note))
     sampler.stop()
 
@@ -738,13 +754,13 @@ def run_ours(args):
                        "parallelism": "replicas only (no exchange step)" if world > 1 else "1 GPU",
                        "launch": "back-to-back C-ABI calls on one stream",
                        "pretouch": "each of the %d rotating buffer sets called once before the warm-up (untimed)" % ROTATE,
-                       "timed": "%d back-to-back loops of %d steps, an event between loops; ms_per_step = median loop / steps"
-                                % (len(loops), args.steps)},
+                       "timed": "%d back-to-back blocks of %d loops of %d steps, an event pair per block; "
+                                "ms_per_step = median block / its steps" % (len(loops), block_steps // args.steps, args.steps)},
             "clocks": sampler.summary(headline_window),
             "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps},
             "gpu_launches": int(launches),
-            "gpu_launches_per_step": launches / float(len(loops) * args.steps),
+            "gpu_launches_per_step": launches / float(len(loops) * block_steps),
             "cpu_baseline": cpu,
             "roofline": {"bound": "hbm", "achieved": per_launch_gbs, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": per_launch_gbs / peaks["hbm_gbs"],

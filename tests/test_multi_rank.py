@@ -93,7 +93,8 @@ def test_gpus_n_without_a_launcher_environment_starts_the_ranks_itself():
 def test_loop_count_and_spread():
     sys.path.insert(0, ROOT)
     import bench
-    assert bench.loop_count(0.25e-3) == 200            # 20 steps of 12.5 us: 200 loops make 50 ms
+    assert bench.loop_count(0.25e-3) == 200            # blocks of 0.25 ms: 200 of them make 50 ms
+    assert bench.loops_per_block(20) == 10 and bench.loops_per_block(1000) == 1 and bench.loops_per_block(7) == 29
     assert bench.loop_count(1.0) == bench.MIN_LOOPS      # long loops: the minimum number of repeats
     assert bench.loop_count(1e-9) == bench.MAX_LOOPS
     s = bench.spread([2e-4, 1e-4, 4e-4], 10)
