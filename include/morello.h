@@ -73,7 +73,8 @@ enum {
  * that would have to grow it while `stream` is being captured returns
  * MORELLO_ERR_WORKSPACE and touches nothing -- size the buffer with an ordinary call
  * on the same shape first, or capture morello_matmul_accum_ws.  The same holds for
- * every entry point below that uses the library's own buffers.
+ * every entry point below that uses the library's own buffers, and the library's first
+ * call on a device (which allocates a 256-byte status block) must come before any capture.
  */
 int morello_matmul_accum(int64_t b, int64_t m, int64_t k, int64_t n,
                          const void* A, const void* B, float* C, void* stream);

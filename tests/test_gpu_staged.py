@@ -23,6 +23,7 @@ SHAPES = [
     (1, 1025, 70, 2051),
     (1, 17, 100, 100),       # small: two chunks of rows on the FMA kernels would cost more
     (2, 260, 72, 1003),      # A is used as it is, C written from registers by CTA pairs, two batches
+    (1, 200, 8200, 303),     # tile kernel with k slices: the reduce launch narrows 304 columns to 303
 ]
 
 
@@ -87,3 +88,39 @@ def test_small_or_few_row_shapes_keep_the_fma_kernels():
         assert mb.morello_select_path(*shape) == mb.MORELLO_PATH_SKINNY
         A, B, C = w.make(*shape, seed=3, ab="int4", c="int8")
         check_full(A, B, C, integer=True, what="%s" % (shape,))
+
+
+def test_growing_a_library_buffer_inside_a_stream_capture_is_refused_cleanly():
+    # The float32 entry point keeps its split operands in a library-owned buffer that grows by
+    # cudaFree + cudaMalloc, which a capturing stream does not allow: the call is refused with
+    # MORELLO_ERR_WORKSPACE before anything touches the device, the capture stays valid, and once an
+    # ordinary call has sized the buffer the same call captures and replays correctly.
+    b, m, k, n = 1, 192, 3136, 3072            # 12 bytes per element of A and B: a buffer no other test needs
+    rng = np.random.default_rng(5)
+    A = rng.integers(-4, 5, size=(b, m, k)).astype(np.float32)
+    B = rng.integers(-4, 5, size=(b, k, n)).astype(np.float32)
+    C = rng.standard_normal((b, m, n)).astype(np.float32)
+    dA, dB, dC = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), torch.from_numpy(C.copy()).cuda()
+    call = mb.lib().morello_matmul_accum_f32
+    mb.morello_device_limits()                 # the library's per-device set-up, outside any capture
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            rc = call(b, m, k, n, dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), side.cuda_stream)
+    assert rc == mb.MORELLO_ERR_WORKSPACE, rc
+    g.replay()                                   # an empty graph: the capture survived the refusal
+    torch.cuda.synchronize()
+    assert torch.equal(dC, torch.from_numpy(C).cuda())
+    mb.morello_matmul_accum_f32(b, m, k, n, dA, dB, dC)          # sizes the buffer
+    torch.cuda.synchronize()
+    want = oracle.matmul_accum_f32(b, m, k, n, A, B, C)
+    assert_bit_exact(dC.cpu().numpy(), want, "float32, integer-valued inputs")
+    g2 = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g2, stream=side):
+            rc = call(b, m, k, n, dA.data_ptr(), dB.data_ptr(), dC.data_ptr(), side.cuda_stream)
+    assert rc == mb.MORELLO_OK
+    g2.replay()
+    torch.cuda.synchronize()
+    assert_bit_exact(dC.cpu().numpy(), oracle.matmul_accum_f32(b, m, k, n, A, B, want), "captured call replayed")
