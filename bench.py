@@ -504,6 +504,29 @@ def bench_layout(torch, mb, idx, iters, peaks, windows, strip=0):
     return rec
 
 
+def cublas_context(torch, shapes):
+    """Context only, never on the library's path and off by default: the time of the vendor
+    library's bf16 GEMM (bf16 output, no accumulate: less work than MatmulAccum's f32
+    read-modify-write of C) on the same shapes and data distribution, same timing loop."""
+    out = []
+    for name, (b, m, k, n), iters in shapes:
+        A = (torch.randn((b, m, k), device="cuda") / k ** 0.5).to(torch.bfloat16)
+        B = (torch.randn((b, k, n), device="cuda") / k ** 0.5).to(torch.bfloat16)
+        C = torch.empty((b, m, n), device="cuda", dtype=torch.bfloat16)
+
+        def step(i):
+            torch.matmul(A, B, out=C)
+
+        loops = [time_calls(torch, step, iters, 3) for _ in range(3)]
+        sec = min(loops) / iters
+        out.append({"name": name, "shape": [b, m, k, n], "us_per_call": sec * 1e6,
+                    "TFLOPs": 2.0 * b * m * k * n / sec / 1e12,
+                    "what": "torch.matmul bf16 -> bf16 (vendor library), context only"})
+        del A, B, C
+        torch.cuda.empty_cache()
+    return out
+
+
 def run_case(args):
     """One configuration alone, device-timed: the command the ncu captures under profiles/
     were taken with, and the unit of single-shape sweeps."""
@@ -715,6 +738,13 @@ def run_ours(args):
                 ("mid_256x8192x8192", (1, 256, 8192, 8192), 100, "one row of pair tiles, long k"),
                 ("gemm_8192_cube", (1, 8192, 8192, 8192), 6, "32 x 32 pair tiles: the tile order's groups of 8 rows keep A and B in L2")):
             extra.append(bench_shape(torch, mb, name, shape, iters, peaks, windows, note))
+    context = None
+    if world == 1 and args.context_cublas:
+        context = cublas_context(torch, [("cfg4_square4096", w.CONFIGS[3].shape, 30),
+                                         ("cfg5_batched", w.CONFIGS[4].shape, 6),
+                                         ("gemm_8192_cube", (1, 8192, 8192, 8192), 6),
+                                         ("mid_256x4096x4096", (1, 256, 4096, 4096), 200),
+                                         ("mid_128x2048x16384", (1, 128, 2048, 16384), 200)])
     sampler.stop()
 
     cpu = None
@@ -737,6 +767,7 @@ def run_ours(args):
         per_launch_gbs = cfg.algorithmic_bytes * args.steps / (sec * 1e9)
         line = {
             "configs": extra,
+            "context_vendor_gemm": context,
             "cpu_baselines": cpu_all,
             "cpu_baselines_note": "the CPU oracle as it stands on this machine's host cores: a baseline, not the target",
             "inputs_crc32": {"A": w.crc32(A), "B0": w.crc32(B0), "C": w.crc32(C)},
@@ -804,6 +835,8 @@ def main(argv=None):
     ap.add_argument("--configs", default="1,3,4,5",
                     help="1-based extra configs to time at --gpus 1 ('' for none)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--context-cublas", action="store_true",
+                    help="also time the vendor library's bf16 GEMM on the GEMM shapes (context only; off by default)")
     ap.add_argument("--case", type=int, default=0,
                     help="time only this 1-based config (with --steps/--warmup calls) and print its record")
     ap.add_argument("--path", default="auto", choices=["auto", "skinny", "tcgen05"],
