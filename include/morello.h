@@ -252,7 +252,8 @@ int morello_select_path(int64_t b, int64_t m, int64_t k, int64_t n);
  * of text for logs: e.g. "tcgen05 gemm_kernel: a CTA pair per 256 x 256 tile, ...".  `text`
  * (host memory, `text_bytes` long, caller-owned) receives at most text_bytes - 1 characters and
  * a terminating NUL.  Enqueues nothing.  Returns MORELLO_OK, MORELLO_ERR_NULL_POINTER for a
- * missing buffer, or MORELLO_ERR_INVALID_SHAPE.
+ * missing buffer, or MORELLO_ERR_INVALID_SHAPE.  With MORELLO_LOG=1 in the environment when the
+ * library is first used, every call that goes through the selector prints this line on stderr.
  */
 int morello_describe_route(int64_t b, int64_t m, int64_t k, int64_t n, char* text, size_t text_bytes);
 

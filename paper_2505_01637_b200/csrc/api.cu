@@ -4,6 +4,7 @@
 #include <atomic>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <mutex>
 
 #include "../../include/morello.h"
@@ -225,6 +226,24 @@ size_t workspace_for(int sms, int path, int knob, int64_t b, int64_t m, int64_t 
   return skinny_workspace(sms, b, m, k, n, B, knob);
 }
 
+// MORELLO_LOG=1 in the environment: every call through the selector prints the route it takes
+// (the line morello_describe_route gives for the shape) on stderr.
+void log_route(int path, int64_t b, int64_t m, int64_t k, int64_t n, bool overwrite, int b_layout) {
+  static const bool on = [] {
+    const char* v = getenv("MORELLO_LOG");
+    return v && v[0] && v[0] != '0';
+  }();
+  if (!on) return;
+  char text[256];
+  if (path != MORELLO_PATH_AUTO || b_layout != 0)
+    snprintf(text, sizeof text, "%s", b_layout ? "B column-major or packed: tensor kernels when addressable, else the plain fallback"
+                                               : "forced path");
+  else if (morello_describe_route(b, m, k, n, text, sizeof text) != MORELLO_OK)
+    snprintf(text, sizeof text, "(no route)");
+  fprintf(stderr, "morello: %s b=%lld m=%lld k=%lld n=%lld -> %s\n", overwrite ? "matmul" : "matmul_accum",
+          (long long)b, (long long)m, (long long)k, (long long)n, text);
+}
+
 int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const void* A,
         const void* B, float* C, void* workspace, size_t workspace_bytes, bool own_scratch,
         void* stream, bool overwrite = false, int b_layout = 0,
@@ -232,6 +251,7 @@ int run(int path, int split_k, int64_t b, int64_t m, int64_t k, int64_t n, const
   bool empty = false;
   int rc = validate(b, m, k, n, A, B, C, &empty);
   if (rc != MORELLO_OK) return rc;
+  log_route(path, b, m, k, n, overwrite, b_layout);
   if (split_k < 0) return MORELLO_ERR_INVALID_SHAPE;
   if (workspace && reinterpret_cast<uintptr_t>(workspace) % 16) return MORELLO_ERR_MISALIGNED;
 

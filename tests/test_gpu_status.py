@@ -36,3 +36,20 @@ def test_selftest_rejects_limits_out_of_range():
         with pytest.raises(mb.MorelloError) as e:
             mb.morello_selftest_wait_timeout(bad)
         assert e.value.status == mb.MORELLO_ERR_INVALID_SHAPE
+
+
+def test_morello_log_prints_the_route_of_every_call():
+    import os, subprocess, sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = ("import sys; sys.path.insert(0, %r); import torch\n"
+            "from paper_2505_01637_b200 import binding as mb\n"
+            "a = torch.zeros(16 * 2048, dtype=torch.int16, device='cuda'); b = torch.zeros(2048 * 1024, dtype=torch.int16, device='cuda')\n"
+            "c = torch.zeros(16 * 1024, device='cuda')\n"
+            "mb.morello_matmul_accum(1, 16, 2048, 1024, a, b, c); mb.morello_matmul(1, 1, 2048, 1024, a, b, c); torch.cuda.synchronize()\n") % root
+    run = subprocess.run([sys.executable, "-c", code], env=dict(os.environ, MORELLO_LOG="1"), capture_output=True,
+                         text=True, timeout=300)
+    assert run.returncode == 0, run.stderr[-2000:]
+    lines = [l for l in run.stderr.splitlines() if l.startswith("morello: ")]
+    assert len(lines) == 2
+    assert lines[0].startswith("morello: matmul_accum b=1 m=16 k=2048 n=1024 -> tcgen05 swap_kernel")
+    assert lines[1].startswith("morello: matmul b=1 m=1 k=2048 n=1024 -> fma ")
