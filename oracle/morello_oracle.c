@@ -18,11 +18,16 @@
  * uint16_t), C[b][m][n] (float).
  *
  * Precision: the paper fixes no summation order (Section 2: the iteration
- * order of a tile loop is undefined), so the oracle is the plain definition:
- * start from (double)C, add the exact products (a bf16 x bf16 product has at
- * most 16 significant bits, exact in double) for p = 0..k-1 in increasing
- * order in double, and round ONCE to float (round-to-nearest-even, the C
- * default) at the end.
+ * order of a tile loop is undefined; Section 2.2 says only that MatmulAccum
+ * accumulates into its output), so the oracle is the plain definition: add the
+ * exact products (a bf16 x bf16 product has at most 16 significant bits, exact
+ * in double) for p = 0..k-1 in increasing order in double, starting from zero,
+ * then add (double)C, and round ONCE to float (round-to-nearest-even, the C
+ * default).  C comes last because a double has 53 bits: a sum that starts
+ * from C loses low bits of C as soon as a partial sum exceeds 2^29 |C|, and
+ * does not get them back when the products cancel (exact rational arithmetic
+ * finds such elements in long sums of small integers); with C last the sum of
+ * integer-valued products is exact and C enters with one rounding.
  *
  * Pins (tests/test_oracle_pins.py): exact rational brute force on tiny
  * shapes, closed forms, identity / zero / one-hot operands, the accumulate
@@ -55,11 +60,11 @@ void oracle_matmul_accum_naive(int64_t b, int64_t m, int64_t k, int64_t n,
     for (int64_t bb = 0; bb < b; ++bb)
         for (int64_t i = 0; i < m; ++i)
             for (int64_t j = 0; j < n; ++j) {
-                double s = (double)C[(bb * m + i) * n + j];
+                double s = 0.0;
                 for (int64_t p = 0; p < k; ++p)
                     s += bf16_to_double(A[(bb * m + i) * k + p]) *
                          bf16_to_double(B[(bb * k + p) * n + j]);
-                C[(bb * m + i) * n + j] = (float)s;
+                C[(bb * m + i) * n + j] = (float)((double)C[(bb * m + i) * n + j] + s);
             }
 }
 
@@ -80,7 +85,7 @@ static void oracle_row(int64_t bb, int64_t i, int64_t m, int64_t k, int64_t n,
                        const float *Cin_row, float *Cout_row, double *T_row,
                        double *s)
 {
-    for (int64_t j = j0; j < j1; ++j) s[j - j0] = (double)Cin_row[j];
+    for (int64_t j = j0; j < j1; ++j) s[j - j0] = 0.0;
     if (T_row) for (int64_t j = j0; j < j1; ++j) T_row[j] = 0.0;
     for (int64_t p = 0; p < k; ++p) {
         const double a = bf16_to_double(A[(bb * m + i) * k + p]);
@@ -90,7 +95,7 @@ static void oracle_row(int64_t bb, int64_t i, int64_t m, int64_t k, int64_t n,
             for (int64_t j = j0; j < j1; ++j)
                 T_row[j] += fabs(a * bf16_to_double(Brow[j]));
     }
-    for (int64_t j = j0; j < j1; ++j) Cout_row[j] = (float)s[j - j0];
+    for (int64_t j = j0; j < j1; ++j) Cout_row[j] = (float)((double)Cin_row[j] + s[j - j0]);
 }
 
 /*
@@ -199,8 +204,8 @@ void oracle_set_num_threads(int t) { (void)t; }
  *     C[b,i,j]  <-  C[b,i,j] + sum_{p=0}^{k-1} A[b,i,p] * B[b,p,j],   A, B, C float
  *
  * A product of two floats has at most 48 significant bits and is exact in double; the
- * sum starts from (double)C, runs over p in increasing order in double and is rounded
- * once to float.  T (may be NULL) receives sum_p |A*B|.  Rows are independent and are
+ * sum starts from zero, runs over p in increasing order in double, (double)C is added
+ * last and the result is rounded once to float.  T (may be NULL) receives sum_p |A*B|.  Rows are independent and are
  * handed to host threads.  Returns 0, or -1 if a row buffer could not be allocated.
  */
 int oracle_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n,
@@ -220,7 +225,7 @@ int oracle_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n,
                 const int64_t bb = r / m;
                 float *Crow = C + r * n;
                 double *Trow = T ? T + r * n : NULL;
-                for (int64_t j = 0; j < n; ++j) s[j] = (double)Crow[j];
+                for (int64_t j = 0; j < n; ++j) s[j] = 0.0;
                 if (Trow) for (int64_t j = 0; j < n; ++j) Trow[j] = 0.0;
                 for (int64_t p = 0; p < k; ++p) {
                     const double a = (double)A[r * k + p];
@@ -228,7 +233,7 @@ int oracle_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n,
                     for (int64_t j = 0; j < n; ++j) s[j] += a * (double)Brow[j];
                     if (Trow) for (int64_t j = 0; j < n; ++j) Trow[j] += fabs(a * (double)Brow[j]);
                 }
-                for (int64_t j = 0; j < n; ++j) Crow[j] = (float)s[j];
+                for (int64_t j = 0; j < n; ++j) Crow[j] = (float)((double)Crow[j] + s[j]);
             }
         }
         free(s);
@@ -242,8 +247,8 @@ int oracle_matmul_accum_f32(int64_t b, int64_t m, int64_t k, int64_t n,
  *
  *     C[b,i,j]  <-  C[b,i,j] + sum_{p=0}^{k-1} A[b,i,p] * Bt[b,j,p],   Bt[b][n][k]
  *
- * Same arithmetic as above (double accumulation of exact products in increasing p, one
- * rounding); only the indexing of the right-hand side differs.
+ * Same arithmetic as above (double accumulation of exact products in increasing p, C added
+ * last, one rounding); only the indexing of the right-hand side differs.
  */
 void oracle_matmul_accum_bt(int64_t b, int64_t m, int64_t k, int64_t n,
                             const uint16_t *A, const uint16_t *Bt, float *C)
@@ -252,11 +257,11 @@ void oracle_matmul_accum_bt(int64_t b, int64_t m, int64_t k, int64_t n,
     for (int64_t r = 0; r < b * m; ++r) {
         const int64_t bb = r / m;
         for (int64_t j = 0; j < n; ++j) {
-            double s = (double)C[r * n + j];
+            double s = 0.0;
             const uint16_t *col = Bt + (bb * n + j) * k;
             for (int64_t p = 0; p < k; ++p)
                 s += bf16_to_double(A[r * k + p]) * bf16_to_double(col[p]);
-            C[r * n + j] = (float)s;
+            C[r * n + j] = (float)((double)C[r * n + j] + s);
         }
     }
 }
@@ -274,7 +279,7 @@ void oracle_matmul_accum_bt(int64_t b, int64_t m, int64_t k, int64_t n,
  *     C[b,i,j]  <-  C[b,i,j] + sum_{p=0}^{k-1} A[b,i,p] * Bp[b][j / s][p][j mod s]
  *
  * Same arithmetic as everywhere above (double accumulation of exact products in increasing p,
- * one rounding); only the indexing of the right-hand side differs.
+ * C added last, one rounding); only the indexing of the right-hand side differs.
  */
 void oracle_matmul_accum_packed_b(int64_t s, int64_t b, int64_t m, int64_t k, int64_t n,
                                   const uint16_t *A, const uint16_t *Bp, float *C)
@@ -284,11 +289,11 @@ void oracle_matmul_accum_packed_b(int64_t s, int64_t b, int64_t m, int64_t k, in
     for (int64_t r = 0; r < b * m; ++r) {
         const int64_t bb = r / m;
         for (int64_t j = 0; j < n; ++j) {
-            double sum = (double)C[r * n + j];
+            double sum = 0.0;
             const uint16_t *col = Bp + ((bb * strips + j / s) * k) * s + (j % s);
             for (int64_t p = 0; p < k; ++p)
                 sum += bf16_to_double(A[r * k + p]) * bf16_to_double(col[p * s]);
-            C[r * n + j] = (float)sum;
+            C[r * n + j] = (float)((double)C[r * n + j] + sum);
         }
     }
 }

@@ -90,6 +90,7 @@ def test_small_or_few_row_shapes_keep_the_fma_kernels():
         check_full(A, B, C, integer=True, what="%s" % (shape,))
 
 
+@pytest.mark.filterwarnings("ignore:The CUDA Graph is empty")
 def test_growing_a_library_buffer_inside_a_stream_capture_is_refused_cleanly():
     # The float32 entry point keeps its split operands in a library-owned buffer that grows by
     # cudaFree + cudaMalloc, which a capturing stream does not allow: the call is refused with

@@ -131,6 +131,42 @@ def test_hand_worked_example():
         assert np.array_equal(run(A, B, C, naive=naive), want)
 
 
+def test_cancelling_products_leave_c_to_the_last_bit():
+    g = _read_golden(os.path.join(GOLDEN, "cancellation_1x1x2x1.txt"))
+    b, m, k, n = (int(v) for v in g["shape"])
+    A = as_bf16(g["A"]).reshape(b, m, k)
+    B = as_bf16(g["B"]).reshape(b, k, n)
+    C = np.array(g["C"], dtype=np.float32).reshape(b, m, n)
+    want = np.array(g["expect"], dtype=np.float32).reshape(b, m, n)
+    assert bits(want)[0, 0, 0] == 0x3F800001
+    for naive in (False, True):
+        assert np.array_equal(bits(run(A, B, C, naive=naive)), bits(want))
+    assert np.array_equal(exact_matmul_accum_bits(A, B, C), bits(want))
+    Bt = np.ascontiguousarray(np.swapaxes(B, 1, 2))
+    assert np.array_equal(bits(oracle.matmul_accum_bt(b, m, k, n, A, Bt, C)), bits(want))
+    assert np.array_equal(bits(oracle.matmul_accum_packed_b(1, b, m, k, n, A, w.pack_b(B, 1), C)), bits(want))
+    got32 = oracle.matmul_accum_f32(b, m, k, n, w.bf16_to_f32(A), w.bf16_to_f32(B), C)
+    assert np.array_equal(bits(got32), bits(want))
+    # the arithmetic that starts the double sum from C does lose the bit: the pin sees it
+    assert not np.array_equal(bits(_mutant(A, B, C, "c_first_double_sum")), bits(want))
+
+
+def test_long_integer_sum_that_cancels_keeps_a_small_c_exactly():
+    # One output element of a seeded 7 x 129 x 11175 x 104 problem with A, B integers in [-4, 4]:
+    # its 11,175 products add up to zero while the partial sums reach into the hundreds, and C is
+    # about 2^-21.  Exact rational arithmetic says the result is C; a double sum that starts from C
+    # drops C's last bit on the way (it needs more than 53 bits there).
+    A, B, C = w.make(7, 129, 11175, 104, seed=1300196, ab="int4", c="normal")
+    a, bcol, c = A[4:5, 31:32, :], B[4:5, :, 87:88], C[4:5, 31:32, 87:88]
+    a, bcol, c = np.ascontiguousarray(a), np.ascontiguousarray(bcol), np.ascontiguousarray(c)
+    assert int((w.bf16_to_f32(a).astype(np.int64).reshape(-1) * w.bf16_to_f32(bcol).astype(np.int64).reshape(-1)).sum()) == 0
+    want = exact_matmul_accum_bits(a, bcol, c)
+    assert np.array_equal(want, bits(c))
+    for naive in (False, True):
+        assert np.array_equal(bits(run(a, bcol, c, naive=naive)), want)
+    assert not np.array_equal(bits(_mutant(a, bcol, c, "c_first_double_sum")), want)
+
+
 def _paper_shapes():
     out = []
     for line in open(os.path.join(GOLDEN, "paper_shapes.txt")):
@@ -302,6 +338,11 @@ def _mutant(A, B, C, kind):
         return (Cd + np.matmul(Af, Bf[:1])).astype(np.float32)
     if kind == "transposed_b":
         return (Cd + np.matmul(Af, np.swapaxes(Bf, 1, 2))).astype(np.float32)
+    if kind == "c_first_double_sum":   # a double sum that starts from C can lose C's low bits
+        s = Cd.copy()
+        for p in range(Af.shape[2]):
+            s = s + Af[:, :, p:p + 1] * Bf[:, p:p + 1, :]
+        return s.astype(np.float32)
     if kind == "f32_preload_sum":   # accumulating in f32 from C is a different rounding
         s = C.copy()
         for p in range(Af.shape[2]):
