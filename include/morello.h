@@ -276,7 +276,10 @@ int morello_describe_route(int64_t b, int64_t m, int64_t k, int64_t n, char* tex
  * bytes) and are added in slice order, then to C, by one more launch: 0 = by shape (only
  * calls whose tiles fill less than half the device and whose k spans at least 32 blocks of 64
  * are cut), 1 = none, 2 .. 8 (fewer are used if a slice would be empty or the sums would
- * exceed 64 MiB).  Returns MORELLO_ERR_UNSUPPORTED_PATH, and
+ * exceed 64 MiB), and ((value / 8192) % 64) is the tile order: tiles are walked in groups of that
+ * many rows of tiles, row-fastest inside a group, so that the tiles in flight share a few rows of
+ * A and a few columns of B (0 = by shape, which is 8; 63 = a whole column of tiles at a time).
+ * Returns MORELLO_ERR_UNSUPPORTED_PATH, and
  * enqueues nothing, when the path cannot run the shape (the tcgen05 path needs
  * k % 8 == 0, n % 8 == 0 and 16-byte-aligned A, B, C) or the value names no tile.
  * workspace may be NULL with workspace_bytes 0 to use the library's own per-device
