@@ -345,7 +345,7 @@ def rotating_sets(in_bytes):
 def bench_calls(torch, mb, name, op, shape, dev_sets, call_one, iters, warmup, peaks, windows, alg_bytes,
                 path_name, extra=None):
     """Device-timed throughput of one arm: `dev_sets` are its rotating operand sets (already on
-    the device), call_one(set) enqueues one call.  Best of three timed loops, the mean beside it."""
+    the device), call_one(set) enqueues one call.  Best of five timed loops, the mean beside it."""
     b, m, k, n = shape
     sets = len(dev_sets)
 
@@ -359,7 +359,7 @@ def bench_calls(torch, mb, name, op, shape, dev_sets, call_one, iters, warmup, p
         step(s)
     per_call = (mb.morello_launch_count() - l0) // sets
     t0 = time.perf_counter()
-    loops = [time_calls(torch, step, iters, warmup if r == 0 else 3) for r in range(3)]
+    loops = [time_calls(torch, step, iters, warmup if r == 0 else 3) for r in range(5)]
     windows.append((t0, time.perf_counter()))
     st, detail = mb.morello_read_device_status()
     if st != 0:
@@ -368,7 +368,7 @@ def bench_calls(torch, mb, name, op, shape, dev_sets, call_one, iters, warmup, p
     flops = 2.0 * b * m * k * n
     gbs, tfl = alg_bytes / sec / 1e9, flops / sec / 1e12
     rec = {"name": name, "op": op, "shape": list(shape), "path": path_name, "us_per_call": sec * 1e6,
-           "us_per_call_mean_of_3_loops": sum(loops) / len(loops) / iters * 1e6,
+           "us_per_call_mean_of_5_loops": sum(loops) / len(loops) / iters * 1e6,
            "GBps": gbs, "TFLOPs": tfl, "iters": iters, "launches_per_call": int(per_call),
            "rotating_sets": sets,
            "frac_hbm_measured": gbs / peaks["hbm_gbs"], "frac_hbm_nominal": gbs / NOMINAL_HBM_GBS,
