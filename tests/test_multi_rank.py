@@ -70,6 +70,11 @@ def test_reference_arm_prints_on_rank_zero_only():
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
     assert line["unit"] == "GB/s" and line["higher_is_better"] is True
+    sys.path.insert(0, ROOT)
+    import bench
+    # both arms name the workload with the same string (the driver compares them)
+    assert line["config"]["workload"] == bench.workload_name(bench.w.CONFIGS[bench.HEADLINE])
+    assert line["metric"] == bench.METRIC
 
 
 def test_gpus_n_without_a_launcher_environment_starts_the_ranks_itself():
