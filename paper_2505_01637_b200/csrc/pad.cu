@@ -55,8 +55,9 @@ __device__ __forceinline__ void pad_one(const PadJob& j, int64_t idx) {
     const uint16_t* at = row + c0;
     if (c0 + 8 <= j.cols_in) {
       // Eight elements inside the row: 32-bit loads where the address allows (the source rows
-      // are only 2-byte aligned), 4 or 5 loads instead of 8.  (Two aligned 16-byte granules and
-      // a funnel shift instead were measured slower.)
+      // are only 2-byte aligned), 4 or 5 loads instead of 8.  (Aligned 16-byte granules with a
+      // funnel shift -- two loads per thread, or one load and the neighbour's granule by warp
+      // shuffles -- were both measured slower.)
       if ((reinterpret_cast<uintptr_t>(at) & 2u) == 0) {
         const uint32_t* q = reinterpret_cast<const uint32_t*>(at);
         w[0] = q[0]; w[1] = q[1]; w[2] = q[2]; w[3] = q[3];
