@@ -65,6 +65,7 @@ MIN_LOOPS = 25          # event-bracketed blocks of K-step loops: at least this 
 MIN_TIMED_SECONDS = 0.05    # ... and until this much work has been timed
 MAX_LOOPS = 4000
 MIN_BLOCK_STEPS = 200   # steps per event pair: an event between launches costs the next its overlap
+ARM_IDLE_SECONDS = 0.5  # pause before each of the other arms, so that none inherits its predecessor's heat
 
 
 def workload_name(cfg):
@@ -358,6 +359,8 @@ def bench_calls(torch, mb, name, op, shape, dev_sets, call_one, iters, warmup, p
     for s in range(sets):                      # every set once: first-use costs stay untimed
         step(s)
     per_call = (mb.morello_launch_count() - l0) // sets
+    torch.cuda.synchronize()
+    time.sleep(ARM_IDLE_SECONDS)               # every arm starts from an idle board, whatever ran before it
     t0 = time.perf_counter()
     loops = [time_calls(torch, step, iters, warmup if r == 0 else 3) for r in range(5)]
     windows.append((t0, time.perf_counter()))
