@@ -19,6 +19,18 @@
  * shape and device, so repeated calls give identical bits.  C is added once,
  * after the sum over k is complete.
  *
+ * Special values follow IEEE 754 as the definition's sum of products does: bf16
+ * subnormal inputs and float32 subnormal sums are kept (no flush to zero), an
+ * infinity or a NaN reaches exactly the elements of C whose sum contains it,
+ * Inf x 0 and Inf - Inf give NaN.  Two exceptions.  (1) When C cannot be
+ * addressed by the TMA engine (n % 8 != 0 or C not 16-byte aligned) and the
+ * tile kernel (more than 64 rows) runs on padded copies, the final C + sum is a
+ * reduction performed in L2, which treats a subnormal C, a subnormal sum and a
+ * subnormal result as zero: an error of at most 2^-126 per element.  (2) The float32
+ * entry point splits its inputs into bf16 terms; an infinite input turns every
+ * result it reaches into NaN (the split forms Inf - Inf) where the definition
+ * gives +-Inf.
+ *
  * Ownership: the caller owns every buffer; the library keeps no reference to
  * them after the enqueued work has run.  C must not overlap A, B or the
  * workspace (not checked).  Unless stated otherwise pointers are DEVICE

@@ -33,8 +33,9 @@
  * shapes, closed forms, identity / zero / one-hot operands, the accumulate
  * invariant, integer exactness against integer matrix products, power-of-two
  * scaling, and agreement with a float64 library contraction.
- * NaN / Inf / subnormal inputs: parity unpinned (they follow IEEE through the
- * C arithmetic below; no test fixes their behaviour).
+ * NaN / Inf / subnormal inputs follow IEEE 754 through the C arithmetic below;
+ * a pin with hand-written expectations (subnormal inputs and sums, infinities
+ * of both signs, NaN operands, Inf x 0, Inf - Inf) fixes that for every variant.
  */
 #include <stdint.h>
 #include <stdlib.h>

@@ -141,6 +141,59 @@ def make_config(index: int, variant: str = "random"):
     raise ValueError(variant)
 
 
+SPECIAL_KINDS = ("subnormal_input", "subnormal_product", "pos_inf", "nan", "inf_minus_inf", "neg_inf")
+
+BF16_MIN_SUBNORMAL = 0x0001     # 2^-133
+BF16_TWO_POW_100 = 0x7180
+BF16_TWO_POW_MINUS_70 = 0x1C80
+BF16_ONE = 0x3F80
+BF16_POS_INF = 0x7F80
+BF16_NEG_INF = 0xFF80
+BF16_QUIET_NAN = 0x7FC0
+
+
+def make_special(m, k, n, seed, first=0):
+    """One batch with IEEE special values planted among small integers (k >= 8, n >= 8).
+
+    Rows 0-5 of B are fixed: row 0 = 2^100, row 1 = 2^-70, row 2 = 1 except a 0 in column 5,
+    row 4 = 1, row 5 = its integers except +Inf in column 6 (row 3 keeps its integers).  Row i of A,
+    for i < 6, is zero but for what its kind plants (kind = SPECIAL_KINDS[(i + first) % 6]):
+    the smallest bf16 subnormal at k index 0; 2^-70 at index 1; +Inf at 2; a NaN at 3; +Inf at 2
+    and -Inf at 4; -Inf at 4.  Those rows start from C = 0.  Every later row is ordinary: integers
+    with zeros at k indices 0-4 and a 1 at index 5 (so that it meets B's +Inf with a factor of 1).
+    Returns (A, B, C, kinds) with kinds[i] the row's kind or "ordinary"."""
+    assert k >= 8 and n >= 8
+    A, B, C = make(1, m, k, n, seed, ab="int4", c="int8")
+    A[0, :, 0:5] = 0
+    A[0, :, 5] = BF16_ONE
+    B[0, 0, :] = BF16_TWO_POW_100
+    B[0, 1, :] = BF16_TWO_POW_MINUS_70
+    B[0, 2, :] = BF16_ONE
+    B[0, 2, 5] = 0
+    B[0, 4, :] = BF16_ONE
+    B[0, 5, 6] = BF16_POS_INF
+    kinds = ["ordinary"] * m
+    for i in range(min(m, len(SPECIAL_KINDS))):
+        kind = SPECIAL_KINDS[(i + first) % len(SPECIAL_KINDS)]
+        kinds[i] = kind
+        A[0, i, :] = 0
+        C[0, i, :] = 0
+        if kind == "subnormal_input":
+            A[0, i, 0] = BF16_MIN_SUBNORMAL
+        elif kind == "subnormal_product":
+            A[0, i, 1] = BF16_TWO_POW_MINUS_70
+        elif kind == "pos_inf":
+            A[0, i, 2] = BF16_POS_INF
+        elif kind == "nan":
+            A[0, i, 3] = BF16_QUIET_NAN
+        elif kind == "inf_minus_inf":
+            A[0, i, 2] = BF16_POS_INF
+            A[0, i, 4] = BF16_NEG_INF
+        elif kind == "neg_inf":
+            A[0, i, 4] = BF16_NEG_INF
+    return A, B, C, kinds
+
+
 def crc32(x: np.ndarray) -> int:
     return zlib.crc32(np.ascontiguousarray(x).view(np.uint8).reshape(-1).data) & 0xFFFFFFFF
 

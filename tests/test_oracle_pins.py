@@ -481,3 +481,61 @@ def test_packed_oracle_one_hot_at_a_hand_computed_offset():
     want[0, :, 6] += -3.0 * Av[0, :, 3]
     got = oracle.matmul_accum_packed_b(s, b, m, k, n, as_bf16(Av), as_bf16(Bp), C)
     assert np.array_equal(got, want)
+
+
+# ------------------------------------------------- IEEE special values
+def special_expectation(A, B, C, kinds):
+    """What IEEE 754 arithmetic fixes for the planted inputs, written out by hand: per element
+    either ("bits", pattern) or ("nan",)."""
+    m, k = A.shape[1], A.shape[2]
+    n = B.shape[2]
+    Ai = w.bf16_to_f32(A)[0].astype(np.float64)
+    Bi = w.bf16_to_f32(B)[0].astype(np.float64)
+    POS_INF, NEG_INF = 0x7F800000, 0xFF800000
+    out = {}
+    for i in range(m):
+        for j in range(n):
+            kind = kinds[i]
+            if kind == "ordinary":
+                if j == 6:                         # 1 x (+Inf) joins finite terms
+                    out[i, j] = ("bits", POS_INF)
+                else:                              # integers only: k indices 0-4 of A are zero
+                    total = int(C[0, i, j]) + sum(int(Ai[i, p]) * int(Bi[p, j]) for p in range(5, k))
+                    out[i, j] = ("bits", frac_to_f32_bits(Fraction(total)))
+            elif j == 6:                           # a special row has a zero against B's +Inf
+                out[i, j] = ("nan",)
+            elif kind == "subnormal_input":        # 2^-133 x 2^100
+                out[i, j] = ("bits", frac_to_f32_bits(Fraction(1, 1 << 33)))
+            elif kind == "subnormal_product":      # 2^-70 x 2^-70: a subnormal float32
+                out[i, j] = ("bits", 1 << 9)
+            elif kind == "pos_inf":                # Inf x 1, but Inf x 0 in column 5
+                out[i, j] = ("nan",) if j == 5 else ("bits", POS_INF)
+            elif kind == "neg_inf":                # -Inf x 1
+                out[i, j] = ("bits", NEG_INF)
+            else:                                  # a NaN operand; Inf - Inf
+                out[i, j] = ("nan",)
+    return out
+
+
+@pytest.mark.parametrize("first", [0, 3])
+def test_special_values_follow_ieee(first):
+    m, k, n = 9, 12, 10
+    A, B, C, kinds = w.make_special(m, k, n, seed=97, first=first)
+    assert set(kinds[:6]) == set(w.SPECIAL_KINDS) and kinds[6:] == ["ordinary"] * 3
+    want = special_expectation(A, B, C, kinds)
+    Bt = np.ascontiguousarray(np.swapaxes(B, 1, 2))
+    Af, Bf = w.bf16_to_f32(A), w.bf16_to_f32(B)
+    results = {
+        "row buffered": oracle.matmul_accum(1, m, k, n, A, B, C),
+        "naive": oracle.matmul_accum(1, m, k, n, A, B, C, naive=True),
+        "column-major B": oracle.matmul_accum_bt(1, m, k, n, A, Bt, C),
+        "packed B": oracle.matmul_accum_packed_b(4, 1, m, k, n, A, w.pack_b(B, 4), C),
+        "float32 inputs": oracle.matmul_accum_f32(1, m, k, n, Af, Bf, C),
+    }
+    for name, got in results.items():
+        gb = bits(got)[0]
+        for (i, j), e in want.items():
+            if e[0] == "nan":
+                assert np.isnan(got[0, i, j]), (name, kinds[i], i, j, got[0, i, j])
+            else:
+                assert int(gb[i, j]) == e[1], (name, kinds[i], i, j, hex(int(gb[i, j])), hex(e[1]))
